@@ -1,0 +1,201 @@
+/*
+ * specpv.h -- C ABI of the SpecPV verification hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, the verification attention of SpecPV
+ * (arXiv 2512.02337): tree-masked grouped-query attention of a step's draft-token tree against a
+ * paged long-context KV cache, either over a small PARTIAL cache (sink blocks + top-scored
+ * retrieval blocks + local window + buffer; paper Section 3.2) or over the FULL cache with a
+ * refresh that rebuilds the partial cache (Section 3.3).  Call names follow Algorithm 1 and the
+ * section titles of the paper.
+ *
+ * Conventions that hold for every call unless stated otherwise
+ *   - "device" pointers are CUDA device memory owned by the caller; the library never allocates,
+ *     frees or keeps them.  "host" pointers are ordinary process memory.
+ *   - Calls that launch work take a `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream), enqueue on it and return without synchronising.
+ *   - Return value: SPECPV_OK or an error found by host-side validation; nothing is launched on
+ *     error.  Faults only the device can see (a page id outside the pool, a cache that would
+ *     overflow, a bounded wait that gave up) are recorded in a status word at the head of the
+ *     `workspace`; the offending work item is skipped and the status is read by
+ *     specpv_poll_status().  No kernel traps or spins without a limit.
+ *   - dtype 0 = float32, 1 = bfloat16 for Q, K, V, the caches, the summaries and the output;
+ *     accumulation is float32; scores and log-sum-exp are float32.
+ *   - Every device pointer must be 16-byte aligned; pools should be 128-byte aligned.
+ *
+ * Tensor layouts (row-major, innermost last)
+ *   K/V pool      [n_layers][n_pages][Hkv][bs][d]     a "page" holds bs tokens of all KV heads
+ *   block_table   [batch][max_blocks] int32           logical block of a sequence -> page id
+ *   seq_lens      [batch] int32                       tokens held by the cache for each sequence
+ *   Q, O          [n_layers_in_call][batch][M_max][Hq][d]
+ *   Knew, Vnew    [n_layers_in_call][batch][M_max][Hkv][d]   keys/values of the step's own tokens
+ *   tree_mask     [batch][M_max][W] uint64, W = ceil(M_max/64); bit a of row j: token j sees token a
+ *   q_lens        [batch] int32   rows actually used per sequence (<= M_max); NULL = M_max for all
+ *   LSE           [n_layers_in_call][batch][M_max][Hq] float32 (natural log)
+ *   summaries     kmax, kmin [n_layers][batch][Hkv][max_blocks][d]   (indexed by LOGICAL block)
+ *   scores        [n_layers_in_call][batch][Hkv][max_blocks] float32
+ *   idx           [n_layers_in_call][batch][Hkv][budget_blocks] int32, count [batch] int32
+ * A partial cache is an ordinary specpv_paged_kv (its own pools, table and lengths); sequence
+ * b's partial segment is the first partial_lens[b] tokens reached through its table.
+ */
+#ifndef SPECPV_H
+#define SPECPV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPECPV_OK = 0,
+    SPECPV_ERR_INVALID_ARG = 1,     /* null pointer, misaligned pointer, negative size */
+    SPECPV_ERR_SHAPE = 2,           /* head counts / head_dim / block size outside what is built */
+    SPECPV_ERR_BUDGET = 3,          /* budget_blocks < sink_blocks + local_blocks + 1 */
+    SPECPV_ERR_CAPACITY = 4,        /* a cache, the workspace or M_max too small for the request */
+    SPECPV_ERR_BAD_TREE = 5,        /* parents[] is not a tree in topological order */
+    SPECPV_ERR_BAD_BLOCK_TABLE = 6, /* a page id outside [0, n_pages) (device-detected) */
+    SPECPV_ERR_UNSUPPORTED = 7,     /* valid request the kernels do not cover */
+    SPECPV_ERR_CUDA = 8,            /* a CUDA runtime call failed */
+    SPECPV_ERR_TIMEOUT = 9          /* a bounded device-side wait gave up (device-detected) */
+} specpv_status;
+
+enum { SPECPV_DTYPE_F32 = 0, SPECPV_DTYPE_BF16 = 1 };
+enum { SPECPV_REDUCE_MEAN = 0, SPECPV_REDUCE_MAX = 1, SPECPV_REDUCE_LAST = 2 };
+enum { SPECPV_MODE_FULL = 0, SPECPV_MODE_PARTIAL = 1, SPECPV_MODE_REFRESH = 2 };
+
+/* Geometry and the method's hyper-parameters (paper Appendix "Generation Settings": block 16,
+ * sink 32 tokens, local 128 tokens, buffer 20 + one step's tokens, reduction = mean). */
+typedef struct {
+    int32_t n_layers;      /* layers held by the pools */
+    int32_t n_q_heads;     /* Hq */
+    int32_t n_kv_heads;    /* Hkv; Hq % Hkv == 0, G = Hq / Hkv */
+    int32_t head_dim;      /* d: 64 or 128 */
+    int32_t block_tokens;  /* bs: tokens per page (16, 32 or 64) */
+    int32_t dtype;         /* SPECPV_DTYPE_* */
+    int32_t sink_blocks;   /* always-kept leading blocks (Section 3.2, "sink tokens") */
+    int32_t local_blocks;  /* always-kept trailing blocks (Section 3.2, "local tokens") */
+    int32_t budget_blocks; /* sink + retrieval + local blocks of the partial cache */
+    int32_t buffer_tokens; /* extra room after the budget for partially verified + candidate tokens */
+    int32_t reduce;        /* SPECPV_REDUCE_*: the f of Eq. 3 */
+    int32_t score_mode;    /* 0 = Eq. 2 as printed (max of the two full dot products) */
+    float softmax_scale;   /* 0 => 1/sqrt(head_dim) */
+} specpv_config;
+
+typedef struct {
+    void *k_pool;               /* device, [n_layers][n_pages][Hkv][bs][d] */
+    void *v_pool;               /* device, same shape */
+    const int32_t *block_table; /* device, [batch][max_blocks] */
+    const int32_t *seq_lens;    /* device, [batch] */
+    int32_t batch;
+    int32_t max_blocks;
+    int32_t n_pages;
+    int32_t max_seq_len; /* host-known upper bound of seq_lens[], used only to size grids */
+} specpv_paged_kv;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char *specpv_status_string(specpv_status s);
+
+/* Bytes of device workspace that any call below needs for the given limits.  The first 256 bytes
+ * hold the device status word and must be zeroed once by the caller (cudaMemset) before first use;
+ * the rest is scratch (split-KV partial results, host-call staging) with no state between calls. */
+size_t specpv_workspace_bytes(const specpv_config *cfg, int n_layers_per_call, int max_batch,
+                              int max_seq_len, int M_max);
+
+/* Synchronises `stream`, returns the device-recorded status (SPECPV_OK if none) and clears it.
+ * info[0..3] (host, nullable) receive kernel-specific details of the first fault. */
+specpv_status specpv_poll_status(void *workspace, void *stream, int32_t *info);
+
+/* Section 3.3 / Algorithm 1 "TreeDecode": ancestor-or-self mask of the step's tokens.
+ * parents (host, [n_tree]): tree-relative parent of each node, parents[0] = -1, parents[i] < i.
+ * n_chain: partially verified tokens placed in front of the tree in a refresh (0 otherwise); they
+ * form a chain and the tree root hangs off the chain's last token.
+ * mask (host, [n_chain + n_tree][row_words] uint64, row_words >= ceil(M/64)) is fully overwritten. */
+specpv_status specpv_build_tree_mask(const int32_t *parents, int n_tree, int n_chain,
+                                     uint64_t *mask, int row_words);
+
+/* Section 3.3 third paragraph / Algorithm 1 "SelectMode": SPECPV_MODE_FULL while the context is
+ * shorter than the budget; one REFRESH to initialise the partial cache; PARTIAL afterwards; REFRESH
+ * again when partially verified + candidate tokens exceed the buffer.  Pure host function. */
+int specpv_select_mode(int ctx_len, int budget_tokens, int n_partially_verified, int n_candidates,
+                       int buffer_tokens, int partial_initialised);
+
+/* Eq. 1: (re)compute Kmax/Kmin of the blocks that hold tokens >= tok_begin[b] (device [batch];
+ * NULL = from token 0) for layers [layer0, layer0 + n_layers).  max_blocks_touched bounds how many
+ * trailing blocks per sequence can change (grid size); pass kv->max_blocks for a full rebuild.
+ * Only the valid tokens of a ragged last block enter the max/min. */
+specpv_status specpv_update_block_summaries(const specpv_config *cfg, int layer0, int n_layers,
+                                            const specpv_paged_kv *kv, const int32_t *tok_begin,
+                                            int max_blocks_touched, void *kmax, void *kmin,
+                                            void *workspace, size_t workspace_bytes, void *stream);
+
+/* Eq. 2-3: scores[l][b][h][i] = f_j max(q_j . Kmax_i, q_j . Kmin_i) over the step's query rows of
+ * KV head h's group (all G heads x q_lens[b] tokens; for SPECPV_REDUCE_LAST the G heads of row
+ * last_query[b] (device [batch], NULL = row 0)).  Blocks >= ceil(seq_len/bs) are left untouched. */
+specpv_status specpv_score_blocks(const specpv_config *cfg, int layer0, int n_layers, const void *q,
+                                  const int32_t *q_lens, int M_max, const int32_t *last_query,
+                                  const void *kmax, const void *kmin, const specpv_paged_kv *kv,
+                                  float *scores, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Section 3.2: the retained block set of every (layer, sequence, KV head): sink blocks, the
+ * budget - sink - local best-scored blocks of [sink, nb - local), and the local blocks, written
+ * ascending to idx; count[b] = min(nb, budget_blocks).  Ties go to the lower block index, NaN
+ * ranks last; the result is a pure function of the float32 scores (bit-exact, deterministic). */
+specpv_status specpv_select_partial_kv(const specpv_config *cfg, int n_layers, const float *scores,
+                                       const int32_t *seq_lens, int batch, int max_blocks,
+                                       int32_t *idx, int32_t *count, void *workspace,
+                                       size_t workspace_bytes, void *stream);
+
+/* Section 3.3 ("refresh the partial KV cache"): copy the selected blocks of every layer and KV
+ * head from the full cache into the partial cache in ascending token order and set
+ * partial_lens[b] = (count[b]-1)*bs + valid tokens of the last block; the buffer starts empty. */
+specpv_status specpv_refresh_partial(const specpv_config *cfg, const specpv_paged_kv *full,
+                                     const int32_t *idx, const int32_t *count,
+                                     const specpv_paged_kv *partial, int32_t *partial_lens,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* Section 3.2 / Algorithm 1 "TreeDecode" with KV_in = KV_partial: tree-masked GQA attention of
+ * the step's tokens over the partial segment (sink | retrieval | local | buffer) followed by the
+ * step's own keys under the tree mask.  out (and lse if not NULL) are fully written for rows
+ * < q_lens[b]. */
+specpv_status specpv_verify_partial(const specpv_config *cfg, int layer0, int n_layers, const void *q,
+                                    const void *k_new, const void *v_new, const uint64_t *tree_mask,
+                                    const int32_t *q_lens, int M_max, const specpv_paged_kv *partial,
+                                    void *out, float *lse, void *workspace, size_t workspace_bytes,
+                                    void *stream);
+
+/* Section 3.3 / Algorithm 1 "TreeDecode" with KV_in = KV_full: the same attention over the whole
+ * cache through the block table.  In a refresh the rows are the partially verified chain followed
+ * by the tree (see specpv_build_tree_mask). */
+specpv_status specpv_verify_full(const specpv_config *cfg, int layer0, int n_layers, const void *q,
+                                 const void *k_new, const void *v_new, const uint64_t *tree_mask,
+                                 const int32_t *q_lens, int M_max, const specpv_paged_kv *full,
+                                 void *out, float *lse, void *workspace, size_t workspace_bytes,
+                                 void *stream);
+
+/* The same step with HOST step tensors (q, k_new, v_new, tree_mask, out, lse are host pointers,
+ * ideally pinned): copies the inputs to staging space inside the workspace, runs the attention
+ * (mode = SPECPV_MODE_PARTIAL or SPECPV_MODE_FULL selects only validation), copies out/lse back and
+ * synchronises the stream before returning.  The KV cache stays device-resident state. */
+specpv_status specpv_verify_host(const specpv_config *cfg, int mode, int layer0, int n_layers,
+                                 const void *q_host, const void *k_new_host, const void *v_new_host,
+                                 const uint64_t *tree_mask_host, int M_max, const specpv_paged_kv *kv,
+                                 void *out_host, float *lse_host, void *workspace,
+                                 size_t workspace_bytes, void *stream);
+
+/* Section 3.2 (buffer) / Section 3.3 (removing invalid tokens): append rows accepted[b][0..n) of
+ * Knew/Vnew (device int32 [batch][A_max], n = n_accepted[b] device [batch]) to cache `dst` at token
+ * positions seq_lens[b].., then seq_lens[b] += n (seq_lens is dst->seq_lens, written in place).
+ * Rejected candidates are simply never appended.  If kmax/kmin are not NULL the summaries of the
+ * touched blocks are recomputed.  A sequence whose cache would overflow is skipped and
+ * SPECPV_ERR_CAPACITY recorded in the status word. */
+specpv_status specpv_commit_accepted(const specpv_config *cfg, int layer0, int n_layers,
+                                     const void *k_new, const void *v_new, int M_max,
+                                     const int32_t *accepted, const int32_t *n_accepted, int A_max,
+                                     const specpv_paged_kv *dst, void *kmax, void *kmin,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECPV_H */
