@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecPV verification hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input:
+  refresh step : tree mask -> full verification over the whole cache -> commit of the accepted path
+                 (with block-summary update) -> block scores -> selection -> gather into the partial cache
+  partial step : tree mask -> partial verification over the partial cache -> commit into its buffer
+The cache lengths are put back after every step so that every step sees the same workload.
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per step with all inputs resident in HBM;
+`e2e` is the same step through the host-buffer entry point (step tensors copied from pinned host
+memory and the outputs copied back inside the timed region); `roofline` is measured live for the
+dominant kernel (full-verification attention); `cpu_baseline` times the CPU oracle on a bounded
+sample of the same workload.  `--impl reference` times only the oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2512_02337_b200 import workloads as wl  # noqa: E402
+
+METRIC = "verify_attention_us_per_step"
+ACCEPT_LEN = 4  # tokens committed per step: the paper's mean accept length is 3.3-3.6 (Table 1), plus the root
+
+
+def load_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_state(name: str, device, n_layers=None, budget_blocks=None):
+    """Allocate every buffer of the step once (torch owns device memory; nothing is allocated per step)."""
+    from paper_2512_02337_b200 import binding as B
+    over = {}
+    if budget_blocks is not None:
+        over["budget_blocks"] = budget_blocks
+    w = wl.make_workload(name, device=device, n_layers=n_layers, spare_tokens=64, **over)
+    c = w.cfg
+    L, Hq, Hkv, d, bs, M, batch = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"], w.batch
+    sink, local = wl.sink_local_blocks(bs)
+    cfg = B.make_config(L, Hq, Hkv, d, bs, c["dtype"], sink, local, c["budget_blocks"], c["buffer_tokens"])
+    dt = wl.torch_dtype(c["dtype"])
+    max_len = max(c["ctx"]) + 64
+    st = dict(w=w, cfg=cfg, B=B, L=L, M=M, batch=batch)
+    st["full"] = B.Cache(w.k_pool, w.v_pool, w.block_table, w.seq_lens, max_len)
+    st["ws"] = B.new_workspace(cfg, L, batch, max_len, M, device=device)
+    st["kmax"] = torch.zeros((L, batch, Hkv, w.max_blocks, d), dtype=dt, device=device)
+    st["kmin"] = torch.zeros_like(st["kmax"])
+    st["scores"] = torch.zeros((L, batch, Hkv, w.max_blocks), dtype=torch.float32, device=device)
+    st["idx"] = torch.zeros((L, batch, Hkv, cfg.budget_blocks), dtype=torch.int32, device=device)
+    st["count"] = torch.zeros(batch, dtype=torch.int32, device=device)
+    ppb = cfg.budget_blocks + (cfg.buffer_tokens + bs - 1) // bs + 1
+    pk = torch.zeros((L, batch * ppb, Hkv, bs, d), dtype=dt, device=device)
+    ptable = torch.arange(batch * ppb, dtype=torch.int32, device=device).reshape(batch, ppb).contiguous()
+    st["plens"] = torch.zeros(batch, dtype=torch.int32, device=device)
+    st["partial"] = B.Cache(pk, torch.zeros_like(pk), ptable, st["plens"], cfg.budget_blocks * bs + cfg.buffer_tokens)
+    st["out"] = torch.zeros((L, batch, M, Hq, d), dtype=dt, device=device)
+    st["lse"] = torch.zeros((L, batch, M, Hq), dtype=torch.float32, device=device)
+    W = (M + 63) // 64
+    st["mask_host"] = torch.zeros((batch, M, W), dtype=torch.int64).pin_memory()
+    st["mask"] = torch.zeros((batch, M, W), dtype=torch.int64, device=device)
+    # accepted path of every sequence: a root-to-node path of ACCEPT_LEN tokens
+    acc = np.zeros((batch, 8), dtype=np.int32)
+    for b in range(batch):
+        depth_of = [len(wl.path_to(w.parents[b], n)) for n in range(M)]
+        acc[b, :ACCEPT_LEN] = wl.path_to(w.parents[b], depth_of.index(ACCEPT_LEN))
+    st["accepted"] = torch.from_numpy(acc).to(device)
+    st["n_accepted"] = torch.full((batch,), ACCEPT_LEN, dtype=torch.int32, device=device)
+    st["lens0"] = w.seq_lens.clone()
+    st["last_query"] = torch.zeros(batch, dtype=torch.int32, device=device)
+    # host copies of the step tensors for the end-to-end path
+    st["host"] = {k: getattr(w, k).cpu().pin_memory() for k in ("q", "k_new", "v_new")}
+    st["out_host"] = torch.zeros((L, batch, M, Hq, d), dtype=dt).pin_memory()
+    st["lse_host"] = torch.zeros((L, batch, M, Hq), dtype=torch.float32).pin_memory()
+    # one-time set-up outside the timed region: summaries of the prefilled cache
+    B.specpv_update_block_summaries(cfg, 0, L, st["full"], None, w.max_blocks, st["kmax"], st["kmin"], st["ws"])
+    torch.cuda.synchronize(device)
+    return st
+
+
+def build_masks(st):
+    """a1: tree masks on the host (library routine), then one async copy."""
+    B, w = st["B"], st["w"]
+    mh = st["mask_host"].numpy().view(np.uint64)
+    for b in range(st["batch"]):
+        mh[b] = B.specpv_build_tree_mask(w.parents[b], 0, mh.shape[2])
+    st["mask"].copy_(st["mask_host"], non_blocking=True)
+
+
+def run_step(st, e2e: bool, events=None):
+    B, w, cfg, L, M, ws = st["B"], st["w"], st["cfg"], st["L"], st["M"], st["ws"]
+    full, partial = st["full"], st["partial"]
+    # ---- refresh step
+    mode = B.specpv_select_mode(int(max(w.cfg["ctx"])), cfg.budget_blocks * cfg.block_tokens, 0, M,
+                                cfg.buffer_tokens, 0)
+    assert mode == B.MODE_REFRESH
+    build_masks(st)
+    if events is not None:
+        events[0].record()
+    if e2e:
+        h = st["host"]
+        B.specpv_verify_host(cfg, B.MODE_FULL, 0, L, h["q"], h["k_new"], h["v_new"], st["mask_host"], M, full,
+                             st["out_host"], st["lse_host"], ws)
+    else:
+        B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, st["mask"], None, M, full, st["out"], st["lse"], ws)
+    if events is not None:
+        events[1].record()
+    B.specpv_commit_accepted(cfg, 0, L, w.k_new, w.v_new, M, st["accepted"], st["n_accepted"], 8, full,
+                             st["kmax"], st["kmin"], ws)
+    B.specpv_score_blocks(cfg, 0, L, w.q, None, M, st["last_query"], st["kmax"], st["kmin"], full, st["scores"], ws)
+    B.specpv_select_partial_kv(cfg, L, st["scores"], w.seq_lens, st["batch"], w.max_blocks, st["idx"], st["count"], ws)
+    B.specpv_refresh_partial(cfg, full, st["idx"], st["count"], partial, st["plens"], ws)
+    # ---- partial step
+    build_masks(st)
+    if events is not None:
+        events[2].record()
+    if e2e:
+        B.specpv_verify_host(cfg, B.MODE_PARTIAL, 0, L, h["q"], h["k_new"], h["v_new"], st["mask_host"], M, partial,
+                             st["out_host"], st["lse_host"], ws)
+    else:
+        B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, st["mask"], None, M, partial, st["out"],
+                                st["lse"], ws)
+    if events is not None:
+        events[3].record()
+    B.specpv_commit_accepted(cfg, 0, L, w.k_new, w.v_new, M, st["accepted"], st["n_accepted"], 8, partial, None,
+                             None, ws)
+    # put the lengths back so that the next step sees the same workload
+    w.seq_lens.copy_(st["lens0"], non_blocking=True)
+
+
+def timed_loop(st, steps, warmup, e2e, dist_barrier):
+    dev = st["w"].device
+    for _ in range(warmup):
+        run_step(st, e2e)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    dist_barrier()
+    launches0 = st["B"].specpv_kernel_launches()
+    t0.record()
+    for i in range(steps):
+        run_step(st, e2e, ev[i])
+    t1.record()
+    torch.cuda.synchronize(dev)
+    dist_barrier()
+    total_ms = t0.elapsed_time(t1)
+    full_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    part_ms = [e[2].elapsed_time(e[3]) for e in ev]
+    st_code, info = st["B"].specpv_poll_status(st["ws"])
+    if st_code != 0:
+        raise RuntimeError(f"device status {st_code} {info}")
+    return total_ms / steps, full_ms, part_ms, st["B"].specpv_kernel_launches() - launches0
+
+
+def algorithmic_work(st):
+    """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
+    c = st["w"].cfg
+    es = 2 if c["dtype"] == "bf16" else 4
+    L, Hq, Hkv, d, M = st["L"], c["Hq"], c["Hkv"], c["d"], c["M"]
+    tokens = sum(c["ctx"])
+    kv_bytes = L * tokens * Hkv * 2 * d * es
+    step_bytes = L * st["batch"] * M * (2 * Hq + 2 * Hkv) * d * es
+    R = (Hq // Hkv) * M
+    flops = L * Hkv * 4 * R * d * (tokens + st["batch"] * M)
+    return kv_bytes + step_bytes, flops, L * M * tokens
+
+
+def oracle_sample(st, budget_s=20.0):
+    """Time the CPU oracle (as it stands) on a bounded sample and scale to one step.
+
+    Sample: layer 0, sequence 0, all KV heads, the rows of one root-to-leaf path of the tree, full
+    verification over the whole context plus partial verification over the partial cache; scaled by
+    (tree tokens / path tokens) x layers x sequences (by context share)."""
+    import oracle
+    w, c = st["w"], st["w"].cfg
+    B = st["B"]
+    M = c["M"]
+    depth_of = [len(wl.path_to(w.parents[0], n)) for n in range(M)]
+    path = wl.path_to(w.parents[0], int(np.argmax(depth_of)))
+    kp, vp = wl.to_numpy(w.k_pool[0]), wl.to_numpy(w.v_pool[0])
+    q, kn, vn = (wl.to_numpy(t[0, 0])[path] for t in (w.q, w.k_new, w.v_new))
+    mask = oracle.tree_mask(np.arange(-1, len(path) - 1, dtype=np.int32))
+    table = w.block_table[0].cpu().numpy()
+    sl = int(st["lens0"][0])
+    t0 = time.perf_counter()
+    oracle.tree_attention(q, kn, vn, mask, kp, vp, table, sl)
+    t_full = time.perf_counter() - t0
+    pk, pv = wl.to_numpy(st["partial"].k_pool[0]), wl.to_numpy(st["partial"].v_pool[0])
+    plen = st["cfg"].budget_blocks * c["bs"]
+    t0 = time.perf_counter()
+    oracle.tree_attention(q, kn, vn, mask, pk, pv, st["partial"].block_table[0].cpu().numpy(), plen)
+    t_part = time.perf_counter() - t0
+    scale = (M / len(path)) * st["L"] * (sum(c["ctx"]) / c["ctx"][0])
+    us = (t_full * scale + t_part * (M / len(path)) * st["L"] * st["batch"]) * 1e6
+    sample = (f"layer 0, sequence 0, all {c['Hkv']} KV heads, {len(path)} of {M} tree tokens (one root-to-leaf "
+              f"path): full verify over {sl} tokens {t_full:.2f}s + partial verify over {plen} tokens "
+              f"{t_part:.2f}s; scaled x{M / len(path):.2f} tokens x{st['L']} layers x sequences; attention only")
+    return us, sample, oracle.num_threads()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama_128k", choices=list(wl.CONFIGS))
+    ap.add_argument("--layers", type=int, default=None, help="truncate the layer count (profiling only)")
+    ap.add_argument("--budget-blocks", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    from paper_2512_02337_b200 import build as build_mod
+    if rank == 0 or not (ROOT / "paper_2512_02337_b200" / "lib" / "libspecpv.so").exists():
+        build_mod.build()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        barrier = lambda: dist.barrier()  # noqa: E731
+    else:
+        barrier = lambda: None  # noqa: E731
+
+    st = build_state(args.workload, dev, args.layers, args.budget_blocks)
+    c = st["w"].cfg
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
+    sampler.start()
+    ms_step, full_ms, part_ms, launches = timed_loop(st, args.steps, warmup, False, barrier)
+    clocks = sampler.stop()
+    e2e = None
+    if not args.no_e2e:
+        e2e_ms, _, _, _ = timed_loop(st, args.steps, warmup, True, barrier)
+    if use_dist:
+        import torch.distributed as dist
+        t = torch.tensor([ms_step, e2e_ms if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, e2e_max = float(t[0]), float(t[1])
+        if not args.no_e2e:
+            e2e_ms = e2e_max
+    if rank != 0:
+        return 0
+
+    peaks = load_peaks()
+    bytes_full, flops_full, tok_kv = algorithmic_work(st)
+    full_avg_s = statistics.mean(full_ms) * 1e-3
+    achieved_gbs = bytes_full / full_avg_s / 1e9
+    achieved_tf = flops_full / full_avg_s / 1e12
+    t_hbm = bytes_full / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = flops_full / (peaks["bf16_tflops"] * 1e12)
+    bound = "hbm" if t_hbm >= t_tensor or c["dtype"] != "bf16" else "tensor"
+    roofline = {"kernel": "full-verification attention (attention + split merge)", "bound": bound,
+                "achieved": achieved_gbs if bound == "hbm" else achieved_tf,
+                "peak": peaks["hbm_gbs"] if bound == "hbm" else peaks["bf16_tflops"],
+                "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                "frac": (achieved_gbs / peaks["hbm_gbs"]) if bound == "hbm" else achieved_tf / peaks["bf16_tflops"],
+                "peak_source": peaks["source"], "traffic": None,
+                "launch_us": full_avg_s * 1e6, "bound_us": max(t_hbm, t_tensor) * 1e6,
+                "achieved_gbs": achieved_gbs, "achieved_tflops": achieved_tf,
+                "frac_of_bound": max(t_hbm, t_tensor) / full_avg_s}
+    out = {
+        "metric": METRIC, "value": ms_step * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": c["dtype"], "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {st['L']} layers, Hq {c['Hq']}, Hkv {c['Hkv']}, d {c['d']}, "
+                               f"ctx {c['ctx']}, {c['bs']}-token pages, tree {c['M']} nodes, budget "
+                               f"{st['cfg'].budget_blocks * c['bs']} tokens, batch {st['batch']}",
+                   "step": "refresh step (full verify + commit + scores + select + gather) + partial step "
+                           "(partial verify + commit)",
+                   "l2": "inputs larger than L2 (every step streams all layers' caches)",
+                   "replicas": "replicas only" if world > 1 else "single GPU"},
+        "phases_us": {"full_verify": statistics.mean(full_ms) * 1e3, "partial_verify": statistics.mean(part_ms) * 1e3,
+                      "rest": ms_step * 1e3 - statistics.mean(full_ms) * 1e3 - statistics.mean(part_ms) * 1e3},
+        "tokens_kv_per_s": world * tok_kv / full_avg_s,
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+    }
+    if not args.no_e2e:
+        L, batch, M = st["L"], st["batch"], c["M"]
+        es = 2 if c["dtype"] == "bf16" else 4
+        h2d = 2 * (L * batch * M * (c["Hq"] + 2 * c["Hkv"]) * c["d"] * es + st["mask_host"].numel() * 8)
+        d2h = 2 * (L * batch * M * c["Hq"] * (c["d"] * es + 4))
+        out["e2e"] = {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    if not args.no_cpu_baseline and world == 1:
+        us, sample, cores = oracle_sample(st)
+        out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
+    print(json.dumps(out))
+    return 0
+
+
+def reference_arm(args):
+    """Times the CPU oracle, as it stands, on bounded samples of the workload (no GPU work at all)."""
+    import oracle
+    name = args.workload
+    c = dict(wl.CONFIGS[name])
+    # one layer, a cut of the context: the sample is scaled to the full step below
+    ctx_cut = [min(x, 8192) for x in c["ctx"]]
+    w = wl.make_workload(name, device="cpu", n_layers=1, ctx=ctx_cut)
+    M = c["M"]
+    depth_of = [len(wl.path_to(w.parents[0], n)) for n in range(M)]
+    path = wl.path_to(w.parents[0], int(np.argmax(depth_of)))
+    kp, vp = wl.to_numpy(w.k_pool[0]), wl.to_numpy(w.v_pool[0])
+    q, kn, vn = (wl.to_numpy(t[0, 0])[path] for t in (w.q, w.k_new, w.v_new))
+    mask = oracle.tree_mask(np.arange(-1, len(path) - 1, dtype=np.int32))
+    table = w.block_table[0].numpy()
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oracle.tree_attention(q, kn, vn, mask, kp, vp, table, ctx_cut[0])
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    budget = c["budget_blocks"] * c["bs"]
+    per_token_row = statistics.mean(times) / (ctx_cut[0] + len(path)) / len(path)
+    step_s = per_token_row * M * c["n_layers"] * (sum(c["ctx"]) + len(c["ctx"]) * budget)
+    sample = (f"oracle attention, 1 layer, sequence 0 cut to {ctx_cut[0]} tokens, all KV heads, {len(path)} of {M} "
+              f"tree tokens; scaled linearly in tokens x rows x layers to the full and partial verification of a step")
+    out = {"impl": "reference", "metric": METRIC, "value": step_s * 1e6, "unit": "us", "n_gpus": 1,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": False,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{name} (see the default arm)"},
+           "cpu_baseline": {"value": step_s * 1e6, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
+                            "sample": sample},
+           "e2e": {"value": step_s * 1e6, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

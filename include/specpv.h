@@ -34,7 +34,7 @@
  *   summaries     kmax, kmin [n_layers][batch][Hkv][max_blocks][d]   (indexed by LOGICAL block)
  *   scores        [n_layers_in_call][batch][Hkv][max_blocks] float32
  *   idx           [n_layers_in_call][batch][Hkv][budget_blocks] int32, count [batch] int32
- * A partial cache is an ordinary specpv_paged_kv (its own pools, table and lengths); sequence
+ * A partial cache is an ordinary specpv_paged_kv with its own pools, table and lengths; sequence
  * b's partial segment is the first partial_lens[b] tokens reached through its table.
  */
 #ifndef SPECPV_H
@@ -101,6 +101,9 @@ const char *specpv_status_string(specpv_status s);
  * the rest is scratch (split-KV partial results, host-call staging) with no state between calls. */
 size_t specpv_workspace_bytes(const specpv_config *cfg, int n_layers_per_call, int max_batch,
                               int max_seq_len, int M_max);
+
+/* Number of kernels this library has launched in this process so far (all streams, monotonic). */
+uint64_t specpv_kernel_launches(void);
 
 /* Synchronises `stream`, returns the device-recorded status (SPECPV_OK if none) and clears it.
  * info[0..3] (host, nullable) receive kernel-specific details of the first fault. */

@@ -1,0 +1,153 @@
+"""GPU parity of the whole hot path on the tiny float32 config and on a small bfloat16 shape:
+summaries, scores, selection, gather, partial and full verification, commit -- each compared with the
+CPU oracle through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_02337_b200 import binding as B
+from paper_2512_02337_b200 import workloads as wl
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def run_pipeline(name, n_layers=None, reduce=0, **over):
+    w = wl.make_workload(name, device="cuda", n_layers=n_layers, spare_tokens=256, **over)
+    c = w.cfg
+    L, Hq, Hkv, d, bs, M = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"]
+    batch = w.batch
+    cfg = util.config_for(w, reduce=reduce)
+    full = util.full_cache(w)
+    full.max_seq_len = int(max(c["ctx"])) + 256
+    ws = B.new_workspace(cfg, L, batch, full.max_seq_len, M)
+    dt = wl.torch_dtype(c["dtype"])
+    dev = w.device
+    mask = util.device_masks(w.parents, M)
+    last_query = torch.zeros(batch, dtype=torch.int32, device=dev)
+
+    # ---- Eq. 1 summaries: bit-exact
+    kmax = torch.zeros((L, batch, Hkv, w.max_blocks, d), dtype=dt, device=dev)
+    kmin = torch.zeros_like(kmax)
+    B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax, kmin, ws)
+    # ---- Eq. 2-3 scores
+    scores = torch.full((L, batch, Hkv, w.max_blocks), float("nan"), dtype=torch.float32, device=dev)
+    B.specpv_score_blocks(cfg, 0, L, w.q, None, M, last_query, kmax, kmin, full, scores, ws)
+    # ---- selection
+    idx = torch.full((L, batch, Hkv, cfg.budget_blocks), -7, dtype=torch.int32, device=dev)
+    count = torch.zeros(batch, dtype=torch.int32, device=dev)
+    B.specpv_select_partial_kv(cfg, L, scores, w.seq_lens, batch, w.max_blocks, idx, count, ws)
+    # ---- gather into the partial cache (pages of sequence b: [b*ppb, (b+1)*ppb), identity table)
+    ppb = cfg.budget_blocks + (cfg.buffer_tokens + bs - 1) // bs + 1
+    pk = torch.zeros((L, batch * ppb, Hkv, bs, d), dtype=dt, device=dev)
+    pv = torch.zeros_like(pk)
+    ptable = torch.arange(batch * ppb, dtype=torch.int32, device=dev).reshape(batch, ppb)
+    plens = torch.zeros(batch, dtype=torch.int32, device=dev)
+    partial = B.Cache(pk, pv, ptable, plens, cfg.budget_blocks * bs + cfg.buffer_tokens)
+    B.specpv_refresh_partial(cfg, full, idx, count, partial, plens, ws)
+    # ---- verification
+    out_full = torch.zeros((L, batch, M, Hq, d), dtype=dt, device=dev)
+    lse_full = torch.zeros((L, batch, M, Hq), dtype=torch.float32, device=dev)
+    out_part, lse_part = torch.zeros_like(out_full), torch.zeros_like(lse_full)
+    B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, out_full, lse_full, ws)
+    B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, out_part, lse_part, ws)
+    util.sync_status(ws)
+
+    seq_lens = w.seq_lens.cpu().numpy()
+    table = w.block_table.cpu().numpy()
+    kp, vp = wl.to_numpy(w.k_pool), wl.to_numpy(w.v_pool)
+    qn, knn, vnn = wl.to_numpy(w.q), wl.to_numpy(w.k_new), wl.to_numpy(w.v_new)
+    kmax_g, kmin_g = util.widen_t(kmax), util.widen_t(kmin)
+    scores_g, idx_g, count_g = scores.cpu().numpy(), idx.cpu().numpy(), count.cpu().numpy()
+    pk_g, pv_g, plens_g = wl.to_numpy(pk), wl.to_numpy(pv), plens.cpu().numpy()
+    sink, local = cfg.sink_blocks, cfg.local_blocks
+    for l in range(L):
+        for b in range(batch):
+            sl = int(seq_lens[b])
+            nb = (sl + bs - 1) // bs
+            okmax, okmin = oracle.block_summaries(kp[l], table[b], sl)
+            assert np.array_equal(kmax_g[l, b, :, :nb], okmax) and np.array_equal(kmin_g[l, b, :, :nb], okmin)
+            osc = oracle.block_scores(qn[l, b], okmax, okmin, Hkv, reduce=reduce, last_query=0)
+            np.testing.assert_allclose(scores_g[l, b, :, :nb], osc, rtol=2e-3 if c["dtype"] == "bf16" else 2e-5,
+                                       atol=2e-2 if c["dtype"] == "bf16" else 2e-4)
+            assert np.all(np.isnan(scores_g[l, b, :, nb:]))  # untouched beyond the context
+            n_keep = min(nb, cfg.budget_blocks)
+            assert count_g[b] == n_keep
+            oidx = np.stack([oracle.select(scores_g[l, b, h, :nb].astype(np.float64), sink, local, cfg.budget_blocks)
+                             for h in range(Hkv)])
+            assert np.array_equal(idx_g[l, b, :, :n_keep], oidx)  # bit-exact given the same float32 scores
+            opk, opv = np.zeros_like(pk_g[l]), np.zeros_like(pv_g[l])
+            oplen = oracle.gather(kp[l], vp[l], table[b], sl, oidx, opk, opv, first_page=b * ppb)
+            assert plens_g[b] == oplen
+            first, last = b * ppb, b * ppb + n_keep
+            gk, gv = pk_g[l, first:last].copy(), pv_g[l, first:last].copy()
+            tail = oplen - (n_keep - 1) * bs
+            gk[-1, :, tail:], gv[-1, :, tail:] = 0, 0   # tokens past the ragged end are unspecified
+            assert np.array_equal(gk, opk[first:last]) and np.array_equal(gv, opv[first:last])
+            omask = oracle.tree_mask(w.parents[b])
+            assert np.array_equal(omask, B.specpv_build_tree_mask(w.parents[b]))
+            o_out, o_lse = oracle.tree_attention(qn[l, b], knn[l, b], vnn[l, b], omask, kp[l], vp[l], table[b], sl)
+            util.compare(util.widen_t(out_full[l, b]), o_out, c["dtype"], f"full out l{l} b{b}")
+            np.testing.assert_allclose(lse_full[l, b].cpu().numpy(), o_lse, atol=2e-5 if c["dtype"] == "fp32" else 2e-3)
+            p_out, p_lse = oracle.tree_attention(qn[l, b], knn[l, b], vnn[l, b], omask, opk, opv,
+                                                 ptable[b].cpu().numpy(), oplen)
+            util.compare(util.widen_t(out_part[l, b]), p_out, c["dtype"], f"partial out l{l} b{b}")
+            np.testing.assert_allclose(lse_part[l, b].cpu().numpy(), p_lse, atol=2e-5 if c["dtype"] == "fp32" else 2e-3)
+    return w, cfg, full, partial, ws, (kmax, kmin)
+
+
+def test_tiny_fp32_config_every_step_matches_oracle():
+    run_pipeline("tiny_fp32")
+
+
+@pytest.mark.parametrize("reduce", [1, 2])
+def test_tiny_fp32_other_reductions(reduce):
+    run_pipeline("tiny_fp32", reduce=reduce)
+
+
+def test_small_bf16_llama_shape_pipeline():
+    # the 32K LLaMA geometry cut down to 2 layers and 6K tokens so that the oracle covers every row
+    run_pipeline("llama_32k", n_layers=2, ctx=[6144 + 37], M=60)
+
+
+def test_ragged_batch_shuffled_table_pipeline():
+    run_pipeline("stress_b4", n_layers=1, ctx=[4096 + 5, 4800, 5120 - 1, 5120], M=64)
+
+
+def test_commit_appends_and_updates_summaries():
+    w, cfg, full, partial, ws, (kmax, kmin) = run_pipeline("tiny_fp32")
+    c = w.cfg
+    L, Hkv, d, bs, M = c["n_layers"], c["Hkv"], c["d"], c["bs"], c["M"]
+    dev = w.device
+    path = wl.path_to(w.parents[0], int(np.argmax([len(wl.path_to(w.parents[0], n)) for n in range(M)])))
+    A_max = 8
+    acc = torch.zeros((1, A_max), dtype=torch.int32, device=dev)
+    acc[0, :len(path)] = torch.from_numpy(path).to(dev)
+    n_acc = torch.tensor([len(path)], dtype=torch.int32, device=dev)
+    kp0, vp0 = wl.to_numpy(w.k_pool).copy(), wl.to_numpy(w.v_pool).copy()
+    sl0 = int(w.seq_lens[0])
+    pl0 = int(partial.seq_lens[0])
+    ppk0, ppv0 = wl.to_numpy(partial.k_pool).copy(), wl.to_numpy(partial.v_pool).copy()
+    # full cache (with summaries) and partial cache (buffer append, no summaries)
+    B.specpv_commit_accepted(cfg, 0, L, w.k_new, w.v_new, M, acc, n_acc, A_max, full, kmax, kmin, ws)
+    B.specpv_commit_accepted(cfg, 0, L, w.k_new, w.v_new, M, acc, n_acc, A_max, partial, None, None, ws)
+    util.sync_status(ws)
+    assert int(w.seq_lens[0]) == sl0 + len(path) and int(partial.seq_lens[0]) == pl0 + len(path)
+    table = w.block_table.cpu().numpy()
+    knn, vnn = wl.to_numpy(w.k_new), wl.to_numpy(w.v_new)
+    for l in range(L):
+        new_len = oracle.commit(knn[l, 0], vnn[l, 0], path, kp0[l], vp0[l], table[0], sl0)
+        assert new_len == sl0 + len(path)
+        oracle.commit(knn[l, 0], vnn[l, 0], path, ppk0[l], ppv0[l], partial.block_table[0].cpu().numpy(), pl0)
+        okmax, okmin = oracle.block_summaries(kp0[l], table[0], new_len)
+        nb = (new_len + bs - 1) // bs
+        assert np.array_equal(util.widen_t(kmax[l, 0])[:, :nb], okmax)
+        assert np.array_equal(util.widen_t(kmin[l, 0])[:, :nb], okmin)
+    assert np.array_equal(wl.to_numpy(w.k_pool), kp0) and np.array_equal(wl.to_numpy(w.v_pool), vp0)
+    assert np.array_equal(wl.to_numpy(partial.k_pool), ppk0) and np.array_equal(wl.to_numpy(partial.v_pool), ppv0)
+    # incremental summaries == full recompute
+    kmax2, kmin2 = torch.zeros_like(kmax), torch.zeros_like(kmin)
+    B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax2, kmin2, ws)
+    nb = (sl0 + len(path) + bs - 1) // bs
+    assert torch.equal(kmax[:, :, :, :nb], kmax2[:, :, :, :nb]) and torch.equal(kmin[:, :, :, :nb], kmin2[:, :, :, :nb])

@@ -1,0 +1,86 @@
+"""Test-side helpers: run the CPU oracle on slices of a workload and compare with the CUDA library."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2512_02337_b200 import binding as B
+from paper_2512_02337_b200 import workloads as wl
+
+# tolerances of the floating-point outputs: max-abs and relative RMS, per storage dtype
+TOL = {"fp32": (1e-5, 1e-5), "bf16": (2e-2, 5e-3)}
+
+
+def config_for(w: wl.Workload, **over) -> B.Config:
+    c = w.cfg
+    sink, local = wl.sink_local_blocks(c["bs"])
+    kw = dict(n_layers=c["n_layers"], n_q_heads=c["Hq"], n_kv_heads=c["Hkv"], head_dim=c["d"],
+              block_tokens=c["bs"], dtype=c["dtype"], sink_blocks=sink, local_blocks=local,
+              budget_blocks=c["budget_blocks"], buffer_tokens=c["buffer_tokens"])
+    kw.update(over)
+    return B.make_config(**kw)
+
+
+def full_cache(w: wl.Workload) -> B.Cache:
+    return B.Cache(w.k_pool, w.v_pool, w.block_table, w.seq_lens, int(max(w.cfg["ctx"])))
+
+
+def device_masks(parents: np.ndarray, M_max: int, n_chain: int = 0, device="cuda") -> torch.Tensor:
+    """[batch][M_max][W] uint64 masks built by the library's host routine, as an int64 device tensor."""
+    W = (M_max + 63) // 64
+    rows = []
+    for p in parents:
+        m = B.specpv_build_tree_mask(p, n_chain, W)
+        pad = np.zeros((M_max, W), dtype=np.uint64)
+        pad[: m.shape[0]] = m
+        rows.append(pad)
+    return torch.from_numpy(np.stack(rows).view(np.int64)).to(device)
+
+
+def compare(got: np.ndarray, want: np.ndarray, dtype: str, what: str = ""):
+    """max-abs and relative-RMS check of a floating-point output against the oracle (float64)."""
+    max_abs_tol, rel_rms_tol = TOL[dtype]
+    got = got.astype(np.float64)
+    assert np.all(np.isfinite(got)), f"{what}: non-finite values"
+    err = np.abs(got - want)
+    rel_rms = np.sqrt((err ** 2).mean()) / max(np.sqrt((want ** 2).mean()), 1e-30)
+    assert err.max() <= max_abs_tol, f"{what}: max-abs {err.max():.3e} > {max_abs_tol}"
+    assert rel_rms <= rel_rms_tol, f"{what}: rel-RMS {rel_rms:.3e} > {rel_rms_tol}"
+    return err.max(), rel_rms
+
+
+def widen_t(t: torch.Tensor) -> np.ndarray:
+    return oracle.widen(wl.to_numpy(t))
+
+
+def oracle_attention_rows(q, k_new, v_new, parents, n_chain, rows, k_pool, v_pool, table, seq_len, scale=None):
+    """Oracle attention for a subset of step rows closed under ancestry.
+
+    ``rows`` are indices into the step's tokens (chain tokens first, then tree nodes); the closure
+    under parents is taken, the sub-tree renumbered, and the oracle run on it.  Because a token only
+    sees its ancestors among the step's tokens, its output equals its output in the full step.
+    Returns (closed_rows, out [n][Hq][d], lse [n][Hq])."""
+    n_tree = len(parents)
+    M = n_chain + n_tree
+    comb = np.concatenate([np.arange(-1, n_chain - 1), np.where(np.asarray(parents) < 0, n_chain - 1,
+                                                                np.asarray(parents) + n_chain)]).astype(np.int64)
+    keep = set()
+    for r in rows:
+        a = int(r)
+        while a >= 0 and a not in keep:
+            keep.add(a)
+            a = int(comb[a])
+    closed = np.array(sorted(keep), dtype=np.int64)
+    renum = {int(r): i for i, r in enumerate(closed)}
+    sub_parents = np.array([renum[int(comb[r])] if comb[r] >= 0 else -1 for r in closed], dtype=np.int32)
+    assert M >= len(closed)
+    mask = oracle.tree_mask(sub_parents)
+    out, lse = oracle.tree_attention(q[closed], k_new[closed], v_new[closed], mask, k_pool, v_pool, table,
+                                     seq_len, scale)
+    return closed, out, lse
+
+
+def sync_status(ws: torch.Tensor, expect: int = 0):
+    st, info = B.specpv_poll_status(ws)
+    assert st == expect, f"device status {st} ({B.specpv_status_string(st)}), info {info}"
