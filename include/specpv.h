@@ -18,8 +18,9 @@
  *     overflow, a bounded wait that gave up) are recorded in a status word at the head of the
  *     `workspace`; the offending work item is skipped and the status is read by
  *     specpv_poll_status().  No kernel traps or spins without a limit.
- *   - dtype 0 = float32, 1 = bfloat16 for Q, K, V, the caches, the summaries and the output;
- *     accumulation is float32; scores and log-sum-exp are float32.
+ *   - dtype 0 = float32, 1 = bfloat16 for Q, K, V, the caches, the summaries and the output
+ *     (the output is float32 instead when cfg->out_f32 is set); accumulation is float32; scores
+ *     and log-sum-exp are float32.
  *   - Every device pointer must be 16-byte aligned; pools should be 128-byte aligned.
  *
  * Tensor layouts (row-major, innermost last)
@@ -80,6 +81,8 @@ typedef struct {
     int32_t reduce;        /* SPECPV_REDUCE_*: the f of Eq. 3 */
     int32_t score_mode;    /* 0 = Eq. 2 as printed (max of the two full dot products) */
     float softmax_scale;   /* 0 => 1/sqrt(head_dim) */
+    int32_t out_f32;       /* 1 => the attention output O is written as float32 whatever dtype is
+                              (the accumulator before the final rounding); 0 => O has type dtype */
 } specpv_config;
 
 typedef struct {

@@ -27,6 +27,7 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     if (cfg->budget_blocks < cfg->sink_blocks + cfg->local_blocks + 1) return SPECPV_ERR_BUDGET;
     if (cfg->reduce < 0 || cfg->reduce > 2) return SPECPV_ERR_INVALID_ARG;
     if (cfg->score_mode != 0) return SPECPV_ERR_UNSUPPORTED;
+    if (cfg->out_f32 != 0 && cfg->out_f32 != 1) return SPECPV_ERR_INVALID_ARG;
     if (!(cfg->softmax_scale >= 0.f) || isinf(cfg->softmax_scale)) return SPECPV_ERR_INVALID_ARG;
     g->n_layers = cfg->n_layers;
     g->Hq = cfg->n_q_heads;
@@ -36,6 +37,8 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     g->bs = cfg->block_tokens;
     g->dtype = cfg->dtype;
     g->es = cfg->dtype == SPECPV_DTYPE_F32 ? 4 : 2;
+    g->out_f32 = (cfg->out_f32 != 0 || cfg->dtype == SPECPV_DTYPE_F32) ? 1 : 0;
+    g->out_es = g->out_f32 ? 4 : 2;
     g->sink_blocks = cfg->sink_blocks;
     g->local_blocks = cfg->local_blocks;
     g->budget_blocks = cfg->budget_blocks;
@@ -62,7 +65,7 @@ StagingPlan plan_staging(const Geometry& g, int n_layers_per_call, int batch, in
     s.k_new = off;  off += round_up(rows * g.Hkv * g.d * g.es, 256);
     s.v_new = off;  off += round_up(rows * g.Hkv * g.d * g.es, 256);
     s.mask = off;   off += round_up((size_t)batch * M_max * ((M_max + 63) / 64) * sizeof(uint64_t), 256);
-    s.out = off;    off += round_up(rows * g.Hq * g.d * g.es, 256);
+    s.out = off;    off += round_up(rows * g.Hq * g.d * g.out_es, 256);
     s.lse = off;    off += round_up(rows * g.Hq * sizeof(float), 256);
     s.total = off;
     return s;
@@ -324,7 +327,8 @@ SPECPV_EXPORT specpv_status specpv_verify_host(const specpv_config* cfg, int mod
                        lse_host ? reinterpret_cast<float*>(stage + sp.lse) : nullptr, workspace,
                        w.partial_off + w.partial_bytes, stream, mode == SPECPV_MODE_PARTIAL);
     if (st != SPECPV_OK) return st;
-    if (cudaMemcpyAsync(out_host, stage + sp.out, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SPECPV_ERR_CUDA;
+    if (cudaMemcpyAsync(out_host, stage + sp.out, rows * g.Hq * g.d * g.out_es, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return SPECPV_ERR_CUDA;
     if (lse_host && cudaMemcpyAsync(lse_host, stage + sp.lse, rows * g.Hq * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return SPECPV_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return SPECPV_ERR_CUDA;

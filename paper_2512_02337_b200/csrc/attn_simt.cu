@@ -54,7 +54,7 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-template <typename T, int D>
+template <typename T, typename TO, int D>
 __global__ void __launch_bounds__(kThreads) attn_simt_kernel(SimtParams p) {
     constexpr int CPL = D / 32;  // channels per lane
     extern __shared__ float smem[];
@@ -197,10 +197,10 @@ __global__ void __launch_bounds__(kThreads) attn_simt_kernel(SimtParams p) {
             if (p.n_splits == 1) {
                 const int j = r / p.G, g = r % p.G;
                 const size_t row = ((size_t)lb * p.M_max + j) * p.Hq + h * p.G + g;
-                T* o = reinterpret_cast<T*>(p.out) + row * D;
+                TO* o = reinterpret_cast<TO*>(p.out) + row * D;
                 float inv = 1.f / l_run[i];
 #pragma unroll
-                for (int c = 0; c < CPL; ++c) o[lane + 32 * c] = from_float<T>(acc[i][c] * inv);
+                for (int c = 0; c < CPL; ++c) o[lane + 32 * c] = from_float<TO>(acc[i][c] * inv);
                 if (p.lse && lane == 0) p.lse[row] = m_run[i] + logf(l_run[i]);
             } else {
                 const size_t prow = (((size_t)lb * p.Hkv + h) * p.n_splits + split) * R_max + r;
@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kThreads) attn_simt_kernel(SimtParams p) {
 
 // Log-sum-exp merge of the per-split partial results: grid = (R_max rows, KV heads, layers x seqs),
 // one thread per channel.
-template <typename T, int D>
+template <typename TO, int D>
 __global__ void __launch_bounds__(D) merge_splits_kernel(SimtParams p) {
     const int r = blockIdx.x, h = blockIdx.y, lb = blockIdx.z, c = threadIdx.x;
     const int b = lb % p.batch;
@@ -239,22 +239,22 @@ __global__ void __launch_bounds__(D) merge_splits_kernel(SimtParams p) {
     }
     const int j = r / p.G, g = r % p.G;
     const size_t row = ((size_t)lb * p.M_max + j) * p.Hq + h * p.G + g;
-    reinterpret_cast<T*>(p.out)[row * D + c] = from_float<T>(o / l_all);
+    reinterpret_cast<TO*>(p.out)[row * D + c] = from_float<TO>(o / l_all);
     if (p.lse && c == 0) p.lse[row] = m_all + logf(l_all);
 }
 
-template <typename T, int D>
+template <typename T, typename TO, int D>
 specpv_status launch_typed(const AttnArgs& a, SimtParams& p, cudaStream_t stream) {
     const size_t smem = (size_t)(kTile * (D + 1) + kTile * D + kRowsPerPass * D) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, TO, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return SPECPV_ERR_CUDA;
     dim3 grid(p.n_splits, a.g.Hkv, a.n_layers * a.batch);
-    attn_simt_kernel<T, D><<<grid, kThreads, smem, stream>>>(p);
+    attn_simt_kernel<T, TO, D><<<grid, kThreads, smem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
     if (p.n_splits > 1) {
         dim3 mgrid(a.M_max * a.g.G, a.g.Hkv, a.n_layers * a.batch);
-        merge_splits_kernel<T, D><<<mgrid, D, 0, stream>>>(p);
+        merge_splits_kernel<TO, D><<<mgrid, D, 0, stream>>>(p);
         if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
         count_launch();
     }
@@ -290,11 +290,14 @@ specpv_status launch_attention_simt(const AttnArgs& a, cudaStream_t stream) {
     p.part_ml = reinterpret_cast<float*>(ws + (size_t)base * n_splits * R_max * a.g.d * sizeof(float));
 
     if (a.g.dtype == SPECPV_DTYPE_F32) {
-        if (a.g.d == 64) return launch_typed<float, 64>(a, p, stream);
-        if (a.g.d == 128) return launch_typed<float, 128>(a, p, stream);
+        if (a.g.d == 64) return launch_typed<float, float, 64>(a, p, stream);
+        if (a.g.d == 128) return launch_typed<float, float, 128>(a, p, stream);
+    } else if (a.g.out_f32) {
+        if (a.g.d == 64) return launch_typed<__nv_bfloat16, float, 64>(a, p, stream);
+        if (a.g.d == 128) return launch_typed<__nv_bfloat16, float, 128>(a, p, stream);
     } else {
-        if (a.g.d == 64) return launch_typed<__nv_bfloat16, 64>(a, p, stream);
-        if (a.g.d == 128) return launch_typed<__nv_bfloat16, 128>(a, p, stream);
+        if (a.g.d == 64) return launch_typed<__nv_bfloat16, __nv_bfloat16, 64>(a, p, stream);
+        if (a.g.d == 128) return launch_typed<__nv_bfloat16, __nv_bfloat16, 128>(a, p, stream);
     }
     return SPECPV_ERR_SHAPE;
 }

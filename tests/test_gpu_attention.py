@@ -44,14 +44,19 @@ def run_case(dtype, Hq, Hkv, d, bs, ctx, Ms, depth=4, branch=3, n_chain=0, n_lay
         masks[b, :m.shape[0]] = m
     q_lens = torch.tensor([m + n_chain for m in Ms], dtype=torch.int32, device=dev)
     seq_lens = torch.tensor(ctx, dtype=torch.int32, device=dev)
-    cfg = B.make_config(n_layers, Hq, Hkv, d, bs, dtype, 1, 1, 3, bs * max_blocks)
+    cfg = B.make_config(n_layers, Hq, Hkv, d, bs, dtype, 1, 1, 3, bs, out_f32=1)
     cache = B.Cache(k_pool, v_pool, torch.from_numpy(table).to(dev), seq_lens, max(ctx))
     ws = B.new_workspace(cfg, n_layers, batch, max(max(ctx), 1), M_max)
-    out = torch.full((n_layers, batch, M_max, Hq, d), 77.0, dtype=dt, device=dev)
+    out = torch.full((n_layers, batch, M_max, Hq, d), 77.0, dtype=torch.float32, device=dev)
     lse = torch.full((n_layers, batch, M_max, Hq), 77.0, dtype=torch.float32, device=dev)
     fn = B.specpv_verify_partial if partial_entry else B.specpv_verify_full
-    fn(cfg, 0, n_layers, q, k_new, v_new, torch.from_numpy(masks.view(np.int64)).to(dev), q_lens, M_max, cache,
-       out, lse, ws)
+    mask_dev = torch.from_numpy(masks.view(np.int64)).to(dev)
+    fn(cfg, 0, n_layers, q, k_new, v_new, mask_dev, q_lens, M_max, cache, out, lse, ws)
+    if dtype == "bf16":  # the bfloat16 output is the float32 one, rounded
+        cfg16 = B.make_config(n_layers, Hq, Hkv, d, bs, dtype, 1, 1, 3, bs, out_f32=0)
+        out16 = torch.full((n_layers, batch, M_max, Hq, d), 77.0, dtype=dt, device=dev)
+        fn(cfg16, 0, n_layers, q, k_new, v_new, mask_dev, q_lens, M_max, cache, out16, None, ws)
+        util.same_as_rounded(out16, out)
     util.sync_status(ws)
     kp, vp = wl.to_numpy(k_pool), wl.to_numpy(v_pool)
     qn, knn, vnn = wl.to_numpy(q), wl.to_numpy(k_new), wl.to_numpy(v_new)

@@ -47,11 +47,18 @@ def run_pipeline(name, n_layers=None, reduce=0, **over):
     partial = B.Cache(pk, pv, ptable, plens, cfg.budget_blocks * bs + cfg.buffer_tokens)
     B.specpv_refresh_partial(cfg, full, idx, count, partial, plens, ws)
     # ---- verification
-    out_full = torch.zeros((L, batch, M, Hq, d), dtype=dt, device=dev)
+    out_full = torch.zeros((L, batch, M, Hq, d), dtype=torch.float32, device=dev)
     lse_full = torch.zeros((L, batch, M, Hq), dtype=torch.float32, device=dev)
     out_part, lse_part = torch.zeros_like(out_full), torch.zeros_like(lse_full)
     B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, out_full, lse_full, ws)
     B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, out_part, lse_part, ws)
+    if c["dtype"] == "bf16":  # the bfloat16 output is the float32 one, rounded
+        cfg16 = util.config_for(w, reduce=reduce, out_f32=0)
+        o16f, o16p = torch.zeros_like(out_full, dtype=dt), torch.zeros_like(out_full, dtype=dt)
+        B.specpv_verify_full(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, o16f, None, ws)
+        B.specpv_verify_partial(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, o16p, None, ws)
+        util.same_as_rounded(o16f, out_full)
+        util.same_as_rounded(o16p, out_part)
     util.sync_status(ws)
 
     seq_lens = w.seq_lens.cpu().numpy()
