@@ -74,10 +74,10 @@ StagingPlan plan_staging(const Geometry& g, int n_layers_per_call, int batch, in
 WorkspacePlan plan_workspace(const Geometry& g, int n_layers_per_call, int max_batch, int M_max) {
     WorkspacePlan w{};
     const size_t base = (size_t)g.Hkv * n_layers_per_call * max_batch;
-    const size_t R_pad = round_up((size_t)M_max * g.G, 128);
+    const size_t R_pad = round_up((size_t)M_max * g.G, 256);
     w.partial_off = kStatusBytes;
-    // room for kTargetCtas + base split results of R_pad rows of (d + 2) floats
-    w.partial_bytes = round_up((kTargetCtas + base) * R_pad * (g.d + 2) * sizeof(float), 256);
+    // room for kMaxSplitCtas + base split results of R_pad rows of (d + 2) floats
+    w.partial_bytes = round_up((kMaxSplitCtas + base) * R_pad * (g.d + 2) * sizeof(float), 256);
     w.staging_off = w.partial_off + w.partial_bytes;
     w.staging_bytes = plan_staging(g, n_layers_per_call, max_batch, M_max).total;
     w.total = w.staging_off + w.staging_bytes;

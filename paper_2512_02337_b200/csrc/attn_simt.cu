@@ -272,7 +272,8 @@ specpv_status launch_attention_simt(const AttnArgs& a, cudaStream_t stream) {
     p.Hq = a.g.Hq; p.Hkv = a.g.Hkv; p.G = a.g.G; p.bs = a.g.bs; p.max_blocks = a.max_blocks; p.n_pages = a.n_pages;
     p.scale = a.g.scale;
 
-    // split the KV range so that the launch has about kTargetCtas CTAs, as far as the workspace allows
+    // split the KV range so that the launch has about two CTAs per SM, as far as the workspace allows
+    constexpr int kTargetCtas = 2 * 148;
     const int base = a.g.Hkv * a.n_layers * a.batch;
     const int R_max = a.M_max * a.g.G;
     int n_splits = (kTargetCtas + base - 1) / base;

@@ -1,17 +1,746 @@
-// Tensor-core (tcgen05 / TMEM / TMA) verification attention for bfloat16, d = 128, 64-token pages.
+// Tensor-core verification attention for B200 (sm_100a): bfloat16, head_dim 128, 64-token pages.
+// Tree-masked GQA attention of the step's tokens over a paged cache (paper Section 3.2-3.3,
+// Algorithm 1 "TreeDecode"), used for both the partial and the full cache.
+//
+// One CTA owns one (layer, sequence, KV head, KV split, row group).  All G query heads of the KV
+// head times up to 2*(128/G) step tokens are packed into two 128-row tiles, so QK^T and PV are
+// dense 128x128x128 contractions:
+//   warp 0      TMA producer: Q once, then K and V tiles of 128 tokens (two pages) through the
+//               block table into a ring of 32 KB shared-memory slots (128-byte swizzle)
+//   warp 1      MMA issuer: tcgen05.mma  S_t = Q_t K^T  (both operands in shared memory) and
+//               O_t += P_t V (P read from tensor memory, V MN-major from shared memory)
+//   warps 4-7   softmax of row tile 0, warps 8-11 of row tile 1: one thread per row reads S from
+//               tensor memory, keeps the running max / sum of an online softmax in the log2
+//               domain, writes P (bfloat16) over S, rescales O only when the max grew by > 2^8,
+//               and finally normalises O and writes it out
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each, P_t aliases S_t.
+// With several KV splits the unnormalised (O, m, l) go to the workspace and merge_kernel combines
+// them by log-sum-exp.  Every wait is bounded; a wait that gives up records SPECPV_ERR_TIMEOUT.
+#include <cuda.h>
+#include <math.h>
+
 #include "common.cuh"
 
 namespace specpv {
 
+namespace {
+
+constexpr int kThreadsTc = 384;          // 12 warps
+constexpr int kTileTokens = 128;         // KV tokens per tile (two 64-token pages)
+constexpr int kD = 128;
+constexpr int kPage = 64;
+constexpr int kSlotBytes = 32768;        // one K or V tile: [2 d-halves][128 tokens][64 d] bf16
+constexpr int kStages = 5;
+constexpr int kQBytes = 2 * 32768;       // two row tiles
+constexpr int kSmemBytes = 1024 + kQBytes + kStages * kSlotBytes;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+struct TcParams {
+    CUtensorMap tm_q;      // (d, Hq, tokens)          box (64, G, 128/G)
+    CUtensorMap tm_knew;   // (d, Hkv, tokens)         box (64, 1, 64)
+    CUtensorMap tm_vnew;
+    CUtensorMap tm_kpool;  // (d, rows)                box (64, 64)
+    CUtensorMap tm_vpool;
+    const uint64_t* tree_mask;
+    const int32_t* q_lens;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    void* out;
+    float* lse;
+    float* part_o;   // [lb][Hkv][splits][R_pad][128]
+    float* part_ml;  // [lb][Hkv][splits][R_pad][2]
+    void* workspace;
+    int layer0, batch, M_max, mask_words, Hq, Hkv, G, max_blocks, n_pages;
+    int n_splits, n_row_groups, R_pad, out_f32;
+    uint32_t pool_rows;  // rows of the pool tensor map (an out-of-range row coordinate reads zeros)
+    float scale_log2;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up after about two seconds (or when another thread already gave up), records
+// SPECPV_ERR_TIMEOUT and raises the CTA's abort flag.  Returns false on give-up.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
+                                            int where) {
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((it & 255u) == 255u && global_ns() - t0 > 2000000000ull) {
+            *abort_flag = 1;
+            record_fault(workspace, SPECPV_ERR_TIMEOUT, where, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
+                                          int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, workspace, where);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+
+#define TMEM_LD32(taddr, v)                                                                                         \
+    asm volatile(                                                                                                   \
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                                   \
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                                   \
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"                   \
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),           \
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),     \
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),   \
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])    \
+        : "r"(taddr)                                                                                                \
+        : "memory")
+
+#define TMEM_ST32(taddr, v)                                                                                         \
+    asm volatile(                                                                                                   \
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                             \
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "                                  \
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"                          \
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),       \
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),             \
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),           \
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])            \
+        : "memory")
+
+#define TMEM_ST16(taddr, v)                                                                                         \
+    asm volatile(                                                                                                   \
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "                                                             \
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"                                  \
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),       \
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])              \
+        : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));  // first source -> upper half
+    return r;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+// K-major operand (rows of 128 bytes, 8-row groups 1024 bytes apart):      lbo = 16 B (unused), sbo = 1024 B.
+// MN-major operand (128 contiguous bytes along MN, rows along K 128 bytes apart, 8-row K groups
+// 1024 bytes apart, next 64-element MN chunk `lbo` bytes away):            lbo = chunk stride, sbo = 1024 B.
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128, N = 128.
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);  // B (= V) is MN-major
+
+struct __align__(8) Barriers {
+    uint64_t q_full;
+    uint64_t kv_full[kStages];
+    uint64_t kv_empty[kStages];
+    uint64_t s_full[2];
+    uint64_t p_full[2];
+    uint64_t o_done[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// =================================================================================================
+__global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_constant__ TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the 128-byte swizzle atoms
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ Barriers bars;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x % p.n_splits, rg = blockIdx.x / p.n_splits;
+    const int h = blockIdx.y, lb = blockIdx.z;
+    const int b = lb % p.batch, l = lb / p.batch;
+
+    const int seq_len = max(p.seq_lens[b], 0);
+    int M = p.q_lens ? p.q_lens[b] : p.M_max;
+    M = min(max(M, 0), p.M_max);
+    const int tok_per_tile = 128 / p.G;               // step tokens per 128-row tile
+    const int tok0 = rg * 2 * tok_per_tile;           // first step token of this row group
+    if (tok0 >= M) return;                            // nothing to do (uniform for the CTA)
+    const int n_q_tiles = (M - tok0 > tok_per_tile) ? 2 : 1;
+
+    // KV range of this split: whole 128-token tiles, split evenly over the sequence's tiles
+    const int total_tiles = (seq_len + kTileTokens - 1) / kTileTokens;
+    const int tiles_per_split = (total_tiles + p.n_splits - 1) / p.n_splits;
+    const int tile_begin = min(split * tiles_per_split, total_tiles);
+    const int tile_end = min(tile_begin + tiles_per_split, total_tiles);
+    const bool last_split = split == p.n_splits - 1;
+    const int n_ctx_tiles = tile_end - tile_begin;
+    const int n_tiles = n_ctx_tiles + (last_split ? 1 : 0);  // the last split also attends the step's own tokens
+
+    const uint32_t q_smem = smem_u32(smem);
+    const uint32_t kv_smem = q_smem + kQBytes;
+    volatile int* abort_flag = &bars.abort_flag;
+
+    if (n_tiles == 0) {
+        // an empty split: publish (m = -inf, l = 0) so that the merge ignores it
+        for (int r = threadIdx.x; r < 256; r += kThreadsTc) {
+            const int row = rg * 256 + r;
+            if (row < p.R_pad) {
+                const size_t prow = (((size_t)lb * p.Hkv + h) * p.n_splits + split) * p.R_pad + row;
+                p.part_ml[prow * 2] = -INFINITY;
+                p.part_ml[prow * 2 + 1] = 0.f;
+            }
+        }
+        return;
+    }
+
+    // ---- set-up ------------------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.q_full), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bars.kv_full[s]), 1);
+            mbar_init(smem_u32(&bars.kv_empty[s]), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(smem_u32(&bars.s_full[t]), 1);
+            mbar_init(smem_u32(&bars.p_full[t]), 128);
+            mbar_init(smem_u32(&bars.o_done[t]), 1);
+        }
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars.tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars.tmem_base;
+    // tensor-memory columns: S_t at t*128, O_t at 256 + t*128; P_t aliases S_t (64 columns of bf16 pairs)
+
+    if (warp == 0) {
+        // =========================== TMA producer ================================================
+        if (lane == 0) {
+            const uint32_t qbar = smem_u32(&bars.q_full);
+            mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
+            for (int t = 0; t < n_q_tiles; ++t)
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(q_smem + t * 32768 + half * 16384, &p.tm_q, half * 64, h * p.G,
+                                lb * p.M_max + tok0 + t * tok_per_tile, qbar);
+            const int32_t* table = p.block_table + (size_t)b * p.max_blocks;
+            const long long layer_row0 = (long long)(p.layer0 + l) * p.n_pages;
+            for (int j = 0; j < n_tiles; ++j) {
+                const bool is_new = j >= n_ctx_tiles;
+                int row[2];  // pool row coordinate of the tile's two pages
+                if (!is_new) {
+                    for (int pg = 0; pg < 2; ++pg) {
+                        const int blk = (tile_begin + j) * 2 + pg;
+                        row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
+                        if ((long long)blk * kPage < seq_len && blk < p.max_blocks) {
+                            const int page = table[blk];
+                            if (page < 0 || page >= p.n_pages)
+                                record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
+                            else
+                                row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
+                        }
+                    }
+                }
+                for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
+                    const int use = 2 * j + kv;
+                    const int slot = use % kStages;
+                    const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
+                    if (use >= kStages && !mbar_wait(empty, ((use / kStages) - 1) & 1, abort_flag, p.workspace, 1)) break;
+                    mbar_expect_tx(full, kSlotBytes);
+                    const uint32_t dst = kv_smem + slot * kSlotBytes;
+                    for (int pg = 0; pg < 2; ++pg)
+                        for (int half = 0; half < 2; ++half) {
+                            const uint32_t d = dst + half * 16384 + pg * 8192;
+                            if (is_new)
+                                tma_load_3d(d, kv ? &p.tm_vnew : &p.tm_knew, half * 64, h, lb * p.M_max + pg * 64, full);
+                            else
+                                tma_load_2d(d, kv ? &p.tm_vpool : &p.tm_kpool, half * 64, row[pg], full);
+                        }
+                }
+                if (*abort_flag) break;
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer ==================================================
+        // Issue order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) | PV(0,1) QK(1,1) | ...
+        bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
+        auto issue_qk = [&](int j, int t) {
+            const int slot = (2 * j) % kStages;
+            const uint32_t kbase = kv_smem + slot * kSlotBytes;
+            const uint32_t qbase = q_smem + t * 32768;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
+                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                mma_ss(tmem + t * 128, make_desc(qbase + off, 16, 1024), make_desc(kbase + off, 16, 1024), kIdescQK,
+                       kk > 0);
+            }
+        };
+        auto issue_pv = [&](int j, int t) {
+            const int slot = (2 * j + 1) % kStages;
+            const uint32_t vbase = kv_smem + slot * kSlotBytes;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
+                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, make_desc(vbase + kk * 2048, 16384, 1024),
+                       kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+            }
+        };
+        for (int j = 0; ok && j <= n_tiles; ++j) {
+            if (j < n_tiles) {
+                // K tile of step j
+                const int use = 2 * j;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, abort_flag, p.workspace, 3));
+                if (!ok) break;
+                tc_fence_after();
+            }
+            for (int t = 0; t < n_q_tiles && ok; ++t) {
+                if (j > 0) {
+                    // PV of the previous tile for this row tile
+                    const int jp = j - 1;
+                    if (t == 0) {
+                        const int use = 2 * jp + 1;
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1,
+                                                                abort_flag, p.workspace, 4));
+                        if (!ok) break;
+                        // rows of V past the tile's valid tokens may hold anything: zero them so that
+                        // 0 * garbage cannot produce NaN
+                        const bool jp_new = jp >= n_ctx_tiles;
+                        const int n_valid = jp_new ? M : min(kTileTokens, seq_len - (tile_begin + jp) * kTileTokens);
+                        if (n_valid < kTileTokens) {
+                            uint8_t* v = smem + kQBytes + (size_t)(use % kStages) * kSlotBytes;
+                            const int n_rows = kTileTokens - n_valid;
+                            for (int i = lane; i < n_rows * 2 * 8; i += 32) {
+                                const int chunk = i & 7, half = (i >> 3) & 1, r = n_valid + (i >> 4);
+                                *reinterpret_cast<uint4*>(v + half * 16384 + r * 128 + chunk * 16) = make_uint4(0, 0, 0, 0);
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                        }
+                    }
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.p_full[t]), jp & 1, abort_flag, p.workspace, 5));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        issue_pv(jp, t);
+                        tc_commit(smem_u32(&bars.o_done[t]));
+                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.kv_empty[(2 * jp + 1) % kStages]));
+                    }
+                    __syncwarp();
+                }
+                if (j < n_tiles) {
+                    if (lane == 0) {
+                        issue_qk(j, t);
+                        tc_commit(smem_u32(&bars.s_full[t]));
+                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.kv_empty[(2 * j) % kStages]));
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // =========================== softmax / correction / epilogue ==============================
+        const int t = (warp - 4) >> 2;           // row tile of this warpgroup
+        const int q = warp & 3;                  // TMEM lane quarter this warp may access
+        const int row_in_tile = q * 32 + lane;
+        if (t < n_q_tiles) {
+            const int row = t * 128 + row_in_tile;                 // row within the row group
+            const int tok = tok0 + row / p.G;                      // step token of this row
+            const int g = row % p.G;
+            const bool row_valid = tok < M;
+            const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+            const uint32_t s_addr = tmem + lane_addr + t * 128;
+            const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
+            uint64_t mask_lo = 0, mask_hi = 0;
+            if (row_valid) {
+                const uint64_t* mrow = p.tree_mask + ((size_t)b * p.M_max + tok) * p.mask_words;
+                mask_lo = mrow[0];
+                if (p.mask_words > 1) mask_hi = mrow[1];
+            }
+            float m_run = -INFINITY, l_run = 0.f;
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const bool is_new = j >= n_ctx_tiles;
+                const int n_valid = is_new ? M : min(kTileTokens, seq_len - (tile_begin + j) * kTileTokens);
+                const bool masked = is_new || n_valid < kTileTokens;
+                uint64_t vis_lo = ~0ull, vis_hi = ~0ull;  // visibility of the tile's 128 columns for this row
+                if (masked) {
+                    if (is_new) {
+                        vis_lo = mask_lo;
+                        vis_hi = mask_hi;
+                    }
+                    if (n_valid < 64) {
+                        vis_lo &= (n_valid <= 0) ? 0ull : (~0ull >> (64 - n_valid));
+                        vis_hi = 0;
+                    } else if (n_valid < 128) {
+                        vis_hi &= (n_valid == 64) ? 0ull : (~0ull >> (128 - n_valid));
+                    }
+                }
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, p.workspace, 6));
+                if (!ok) break;
+                tc_fence_after();
+                // pass 1: row maximum of the visible logits
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    TMEM_LD32(s_addr + c * 32, v);
+                    tmem_wait_ld();
+                    const uint32_t bits = (uint32_t)((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        float s = __uint_as_float(v[i]);
+                        if (masked) s = ((bits >> i) & 1u) ? s : -INFINITY;
+                        mx = fmaxf(mx, s);
+                    }
+                }
+                const float m_tile = mx * p.scale_log2;
+                // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger.
+                // The decision is per row, the tensor-memory traffic is warp-wide: if any row of the
+                // warp rescales, all 32 rows pass through it (with a factor of 1 where nothing changes).
+                bool need = false;
+                if (j == 0) {
+                    m_run = m_tile;
+                } else {
+                    need = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
+                }
+                if (__any_sync(0xffffffffu, need)) {
+                    const float factor = !need ? 1.f : (m_run == -INFINITY ? 0.f : ex2(m_run - m_tile));
+                    // O_t must hold every earlier PV before it is rescaled
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag, p.workspace, 7));
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t v[32];
+                        TMEM_LD32(o_addr + c * 32, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * factor);
+                        TMEM_ST32(o_addr + c * 32, v);
+                    }
+                    if (need) {
+                        l_run *= factor;
+                        m_run = m_tile;
+                    }
+                }
+                const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+                // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over S
+                float l_add = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    TMEM_LD32(s_addr + c * 32, v);
+                    tmem_wait_ld();
+                    const uint32_t bits = (uint32_t)((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
+                        float p0 = ex2(fmaf(s0, p.scale_log2, -m_use));
+                        float p1 = ex2(fmaf(s1, p.scale_log2, -m_use));
+                        if (masked) {
+                            p0 = ((bits >> i) & 1u) ? p0 : 0.f;
+                            p1 = ((bits >> (i + 1)) & 1u) ? p1 : 0.f;
+                        }
+                        const uint32_t w = pack_bf16(p0, p1);
+                        pk[i >> 1] = w;
+                        // the row sum is taken over the ROUNDED weights the tensor core will use, so
+                        // that O / l is an exact weighted average of V rows (rounding errors of a
+                        // dominant weight cancel instead of scaling the output)
+                        l_add += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+                    }
+                    // all four chunks of S have been read into registers before P overwrites columns
+                    // [0, 64): chunk c of P lands in columns [16c, 16c + 16), which only overlaps S
+                    // chunks <= c/2 that this thread has already consumed
+                    TMEM_ST16(s_addr + c * 16, pk);
+                }
+                l_run += l_add;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_full[t]));
+            }
+            // ---- epilogue: wait for the last PV, normalise, write out ---------------------------
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), (n_tiles - 1) & 1, abort_flag, p.workspace, 8));
+            if (ok) {
+                tc_fence_after();
+                const bool direct = p.n_splits == 1;
+                const float inv = direct ? 1.f / l_run : 1.f;
+                const size_t out_row = ((size_t)lb * p.M_max + tok) * p.Hq + h * p.G + g;
+                const size_t prow = (((size_t)lb * p.Hkv + h) * p.n_splits + split) * p.R_pad + rg * 256 + row;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    TMEM_LD32(o_addr + c * 32, v);
+                    tmem_wait_ld();
+                    if (!row_valid) continue;
+                    if (!direct) {
+                        uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * kD + c * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    } else if (p.out_f32) {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_row * kD + c * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_float4(__uint_as_float(v[4 * i]) * inv, __uint_as_float(v[4 * i + 1]) * inv,
+                                                 __uint_as_float(v[4 * i + 2]) * inv, __uint_as_float(v[4 * i + 3]) * inv);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_row * kD + c * 32);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(v[8 * i]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+                            w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+                            w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+                            w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+                            dst[i] = w;
+                        }
+                    }
+                }
+                if (row_valid) {
+                    if (direct) {
+                        if (p.lse) p.lse[out_row] = m_run * kLn2 + logf(l_run);
+                    } else {
+                        p.part_ml[prow * 2] = m_run * kLn2;  // natural-log units for the merge
+                        p.part_ml[prow * 2 + 1] = l_run;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (*abort_flag) __nanosleep(200000);  // let copies in flight land before the CTA goes away
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+// Log-sum-exp merge of the KV splits: grid = (R rows, Hkv, layers x seqs), one thread per channel.
+__global__ void __launch_bounds__(kD) merge_tc_kernel(TcParams p) {
+    const int r = blockIdx.x, h = blockIdx.y, lb = blockIdx.z, c = threadIdx.x;
+    const int b = lb % p.batch;
+    int M = p.q_lens ? p.q_lens[b] : p.M_max;
+    M = min(max(M, 0), p.M_max);
+    if (r >= M * p.G) return;
+    const size_t base = ((size_t)lb * p.Hkv + h) * p.n_splits;
+    float m_all = -INFINITY;
+    for (int s = 0; s < p.n_splits; ++s) m_all = fmaxf(m_all, p.part_ml[((base + s) * p.R_pad + r) * 2]);
+    float l_all = 0.f, o = 0.f;
+    for (int s = 0; s < p.n_splits; ++s) {
+        const size_t prow = (base + s) * p.R_pad + r;
+        const float m_s = p.part_ml[prow * 2];
+        if (m_s == -INFINITY) continue;
+        const float w = __expf(m_s - m_all);
+        l_all = fmaf(p.part_ml[prow * 2 + 1], w, l_all);
+        o = fmaf(p.part_o[prow * kD + c], w, o);
+    }
+    const int j = r / p.G, g = r % p.G;
+    const size_t row = ((size_t)lb * p.M_max + j) * p.Hq + h * p.G + g;
+    const float val = o / l_all;
+    if (p.out_f32) reinterpret_cast<float*>(p.out)[row * kD + c] = val;
+    else reinterpret_cast<__nv_bfloat16*>(p.out)[row * kD + c] = __float2bfloat16_rn(val);
+    if (p.lse && c == 0) p.lse[row] = m_all + logf(l_all);
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+bool encode_map(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                const uint32_t* box) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[5], gstride[5];
+    cuuint32_t gbox[5], estride[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        gbox[i] = box[i];
+        estride[i] = 1;
+        if (i > 0) gstride[i - 1] = strides_bytes[i - 1];
+    }
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, gbox,
+              estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 bool attention_tc_supported(const AttnArgs& a) {
-    (void)a;
-    return false;
+    if (a.g.dtype != SPECPV_DTYPE_BF16 || a.g.d != 128 || a.g.bs != 64) return false;
+    if (a.g.G > 128 || (128 % a.g.G) != 0) return false;
+    if (a.M_max > kMaxQTokens) return false;
+    // row coordinates of the pool tensor map must fit in a positive int32
+    const unsigned long long rows = (unsigned long long)a.g.n_layers * a.n_pages * a.g.Hkv * 64ull;
+    if (rows >= 0x7FFFFF00ull) return false;
+    return get_encode_fn() != nullptr;
 }
 
 specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
-    (void)a;
-    (void)stream;
-    return SPECPV_ERR_UNSUPPORTED;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return SPECPV_ERR_CUDA;
+        attr_set = true;
+    }
+    TcParams p{};
+    const int G = a.g.G, Hq = a.g.Hq, Hkv = a.g.Hkv;
+    const uint64_t step_tokens = (uint64_t)a.n_layers * a.batch * a.M_max;
+    {
+        uint64_t dims[3] = {128, (uint64_t)Hq, step_tokens};
+        uint64_t strides[2] = {256, (uint64_t)Hq * 256};
+        uint32_t box[3] = {64, (uint32_t)G, (uint32_t)(128 / G)};
+        if (!encode_map(&p.tm_q, a.q, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
+    }
+    {
+        uint64_t dims[3] = {128, (uint64_t)Hkv, step_tokens};
+        uint64_t strides[2] = {256, (uint64_t)Hkv * 256};
+        uint32_t box[3] = {64, 1, 64};
+        if (!encode_map(&p.tm_knew, a.k_new, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
+        if (!encode_map(&p.tm_vnew, a.v_new, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
+    }
+    const uint64_t pool_rows = (uint64_t)a.g.n_layers * a.n_pages * Hkv * 64ull;
+    {
+        uint64_t dims[2] = {128, pool_rows};
+        uint64_t strides[1] = {256};
+        uint32_t box[2] = {64, 64};
+        if (!encode_map(&p.tm_kpool, a.k_pool, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
+        if (!encode_map(&p.tm_vpool, a.v_pool, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
+    }
+    p.tree_mask = a.tree_mask; p.q_lens = a.q_lens; p.block_table = a.block_table; p.seq_lens = a.seq_lens;
+    p.out = a.out; p.lse = a.lse; p.workspace = a.workspace;
+    p.layer0 = a.layer0; p.batch = a.batch; p.M_max = a.M_max; p.mask_words = a.mask_words;
+    p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.max_blocks = a.max_blocks; p.n_pages = a.n_pages;
+    p.out_f32 = a.g.out_f32;
+    p.pool_rows = (uint32_t)pool_rows;
+    p.scale_log2 = a.g.scale * kLog2e;
+
+    const int R_max = a.M_max * G;
+    p.n_row_groups = (R_max + 255) / 256;
+    p.R_pad = p.n_row_groups * 256;
+    // KV splits: fill the 148 SMs (one CTA each) in whole waves as evenly as the workspace allows
+    const int base = Hkv * a.n_layers * a.batch * p.n_row_groups;
+    const int max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens;
+    const size_t per_split = (size_t)Hkv * a.n_layers * a.batch * p.R_pad * (kD + 2) * sizeof(float);
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 64; ++s) {
+        if (s > 1 && (s > max_tiles / 4 || per_split * s > a.partial_bytes)) break;
+        const long long ctas = (long long)base * s;
+        const double eff = (double)ctas / (double)(((ctas + 147) / 148) * 148);
+        if (eff > best_eff + 0.02) {
+            best_eff = eff;
+            best = s;
+        }
+    }
+    p.n_splits = best;
+    char* ws = reinterpret_cast<char*>(a.workspace) + a.partial_off;
+    p.part_o = reinterpret_cast<float*>(ws);
+    p.part_ml = reinterpret_cast<float*>(ws + (size_t)Hkv * a.n_layers * a.batch * p.n_splits * p.R_pad * kD * sizeof(float));
+
+    dim3 grid(p.n_splits * p.n_row_groups, Hkv, a.n_layers * a.batch);
+    attn_tc_kernel<<<grid, kThreadsTc, kSmemBytes, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+    count_launch();
+    if (p.n_splits > 1) {
+        dim3 mgrid(R_max, Hkv, a.n_layers * a.batch);
+        merge_tc_kernel<<<mgrid, kD, 0, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+        count_launch();
+    }
+    return SPECPV_OK;
 }
 
 }  // namespace specpv

@@ -29,7 +29,7 @@ __device__ __forceinline__ void record_fault(void* workspace, int code, int i0, 
 
 constexpr size_t kStatusBytes = 256;
 constexpr int kMaxQTokens = 128;      // M_max supported by the attention kernels (two mask words)
-constexpr int kTargetCtas = 2 * 148;  // split-KV aims at this many CTAs per launch
+constexpr int kMaxSplitCtas = 8 * 148;  // the workspace holds split-KV partial results of this many CTAs (+ one per head)
 
 // process-wide count of kernel launches (reported by specpv_kernel_launches)
 void count_launch(int n = 1);

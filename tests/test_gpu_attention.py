@@ -68,7 +68,7 @@ def run_case(dtype, Hq, Hkv, d, bs, ctx, Ms, depth=4, branch=3, n_chain=0, n_lay
             o_out, o_lse = oracle.tree_attention(qn[l, b, :m], knn[l, b, :m], vnn[l, b, :m], omask, kp[l], vp[l],
                                                  table[b], ctx[b])
             util.compare(util.widen_t(out[l, b, :m]), o_out, dtype, f"out l{l} b{b}")
-            np.testing.assert_allclose(lse[l, b, :m].cpu().numpy(), o_lse, atol=2e-5 if dtype == "fp32" else 3e-3)
+            np.testing.assert_allclose(lse[l, b, :m].cpu().numpy(), o_lse, atol=2e-5 if dtype == "fp32" else 5e-3)
             # rows past q_lens[b] are not written
             assert torch.all(out[l, b, m:].float() == 77.0)
 

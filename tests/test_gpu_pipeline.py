@@ -96,11 +96,11 @@ def run_pipeline(name, n_layers=None, reduce=0, **over):
             assert np.array_equal(omask, B.specpv_build_tree_mask(w.parents[b]))
             o_out, o_lse = oracle.tree_attention(qn[l, b], knn[l, b], vnn[l, b], omask, kp[l], vp[l], table[b], sl)
             util.compare(util.widen_t(out_full[l, b]), o_out, c["dtype"], f"full out l{l} b{b}")
-            np.testing.assert_allclose(lse_full[l, b].cpu().numpy(), o_lse, atol=2e-5 if c["dtype"] == "fp32" else 2e-3)
+            np.testing.assert_allclose(lse_full[l, b].cpu().numpy(), o_lse, atol=2e-5 if c["dtype"] == "fp32" else 5e-3)
             p_out, p_lse = oracle.tree_attention(qn[l, b], knn[l, b], vnn[l, b], omask, opk, opv,
                                                  ptable[b].cpu().numpy(), oplen)
             util.compare(util.widen_t(out_part[l, b]), p_out, c["dtype"], f"partial out l{l} b{b}")
-            np.testing.assert_allclose(lse_part[l, b].cpu().numpy(), p_lse, atol=2e-5 if c["dtype"] == "fp32" else 2e-3)
+            np.testing.assert_allclose(lse_part[l, b].cpu().numpy(), p_lse, atol=2e-5 if c["dtype"] == "fp32" else 5e-3)
     return w, cfg, full, partial, ws, (kmax, kmin)
 
 
