@@ -89,7 +89,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 
 // Bounded wait: gives up after about two seconds (or when another thread already gave up), records
 // SPECPV_ERR_TIMEOUT and raises the CTA's abort flag.  Returns false on give-up.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
                                             int where) {
     const uint64_t t0 = global_ns();
     for (uint32_t it = 0;; ++it) {
@@ -290,7 +290,9 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t tmem = bars.tmem_base;
     // tensor-memory columns: S_t at t*128, O_t at 256 + t*128; P_t aliases S_t (64 columns of bf16 pairs)
 
+    // Register budget: the control warpgroup (warps 0-3) gives registers to the two softmax warpgroups.
     if (warp == 0) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== TMA producer ================================================
         if (lane == 0) {
             const uint32_t qbar = smem_u32(&bars.q_full);
@@ -337,6 +339,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             }
         }
     } else if (warp == 1) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== MMA issuer ==================================================
         // Issue order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) | PV(0,1) QK(1,1) | ...
         bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
@@ -412,7 +415,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 }
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
         // =========================== softmax / correction / epilogue ==============================
         const int t = (warp - 4) >> 2;           // row tile of this warpgroup
         const int q = warp & 3;                  // TMEM lane quarter this warp may access
@@ -453,21 +459,29 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, p.workspace, 6));
                 if (!ok) break;
                 tc_fence_after();
-                // pass 1: row maximum of the visible logits
-                float mx = -INFINITY;
+                // the whole row of S (128 columns) goes to registers in one round trip
+                uint32_t v[128];
+                TMEM_LD32(s_addr, v);
+                TMEM_LD32(s_addr + 32, (v + 32));
+                TMEM_LD32(s_addr + 64, (v + 64));
+                TMEM_LD32(s_addr + 96, (v + 96));
+                tmem_wait_ld();
+                if (masked) {  // ragged or tree-masked tile: invisible columns become -inf (at most two tiles per CTA)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    TMEM_LD32(s_addr + c * 32, v);
-                    tmem_wait_ld();
-                    const uint32_t bits = (uint32_t)((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float s = __uint_as_float(v[i]);
-                        if (masked) s = ((bits >> i) & 1u) ? s : -INFINITY;
-                        mx = fmaxf(mx, s);
+                    for (int i = 0; i < 128; ++i) {
+                        const uint64_t word = i < 64 ? vis_lo : vis_hi;
+                        if (!((word >> (i & 63)) & 1ull)) v[i] = 0xff800000u;
                     }
                 }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 128; i += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(v[i]));
+                    mx1 = fmaxf(mx1, __uint_as_float(v[i + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(v[i + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(v[i + 3]));
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 const float m_tile = mx * p.scale_log2;
                 // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger.
                 // The decision is per row, the tensor-memory traffic is warp-wide: if any row of the
@@ -486,12 +500,12 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        uint32_t v[32];
-                        TMEM_LD32(o_addr + c * 32, v);
+                        uint32_t o[32];
+                        TMEM_LD32(o_addr + c * 32, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * factor);
-                        TMEM_ST32(o_addr + c * 32, v);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        TMEM_ST32(o_addr + c * 32, o);
                     }
                     if (need) {
                         l_run *= factor;
@@ -499,36 +513,25 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     }
                 }
                 const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over S
-                float l_add = 0.f;
+                // P = 2^(s*scale - m) as bf16 pairs written over S (all of S is already in registers).  The row sum is taken over the ROUNDED weights the
+                // tensor core will use, so that O / l is an exact weighted average of V rows (the rounding
+                // error of a dominant weight cancels instead of scaling the output).
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 nm2 = make_float2(-m_use, -m_use);
+                float2 sum2 = make_float2(0.f, 0.f);
+                // packed in place: word i of P (columns 2i, 2i+1) overwrites v[i], whose own value was
+                // consumed by an earlier pair, so no second register array is needed
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    TMEM_LD32(s_addr + c * 32, v);
-                    tmem_wait_ld();
-                    const uint32_t bits = (uint32_t)((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
-                        float p0 = ex2(fmaf(s0, p.scale_log2, -m_use));
-                        float p1 = ex2(fmaf(s1, p.scale_log2, -m_use));
-                        if (masked) {
-                            p0 = ((bits >> i) & 1u) ? p0 : 0.f;
-                            p1 = ((bits >> (i + 1)) & 1u) ? p1 : 0.f;
-                        }
-                        const uint32_t w = pack_bf16(p0, p1);
-                        pk[i >> 1] = w;
-                        // the row sum is taken over the ROUNDED weights the tensor core will use, so
-                        // that O / l is an exact weighted average of V rows (rounding errors of a
-                        // dominant weight cancel instead of scaling the output)
-                        l_add += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
-                    }
-                    // all four chunks of S have been read into registers before P overwrites columns
-                    // [0, 64): chunk c of P lands in columns [16c, 16c + 16), which only overlaps S
-                    // chunks <= c/2 that this thread has already consumed
-                    TMEM_ST16(s_addr + c * 16, pk);
+                for (int i = 0; i < 64; ++i) {
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])),
+                                                sc2, nm2);
+                    const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
+                    v[i] = w;
+                    sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+                    if (i == 31) TMEM_ST32(s_addr, v);
                 }
+                TMEM_ST32(s_addr + 32, (v + 32));
+                const float l_add = sum2.x + sum2.y;
                 l_run += l_add;
                 tmem_wait_st();
                 tc_fence_before();
