@@ -234,7 +234,10 @@ SPECPV_EXPORT specpv_status specpv_score_blocks(const specpv_config* cfg, int la
     p.q = q; p.q_lens = q_lens; p.last_query = last_query; p.kmax = kmax; p.kmin = kmin; p.seq_lens = kv->seq_lens;
     p.scores = scores; p.layer0 = layer0; p.batch = kv->batch; p.M_max = M_max; p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
     p.bs = g.bs; p.max_blocks = kv->max_blocks; p.reduce = g.reduce;
+    p.workspace = workspace;
     const int max_nb = (kv->max_seq_len + g.bs - 1) / g.bs;
+    if (scores_tc_supported(g.dtype, g.d, g.G, M_max) && aligned16(q) && aligned16(kmax) && aligned16(kmin))
+        return launch_scores_tc(p, n_layers, g.n_layers, max_nb, reinterpret_cast<cudaStream_t>(stream));
     return launch_scores(p, n_layers, max_nb, g.dtype, g.d, reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -24,6 +24,7 @@ struct ScoreParams {
     const void* kmin;
     const int32_t* seq_lens;
     float* scores;
+    void* workspace;
     int layer0, batch, M_max, Hq, Hkv, G, bs, max_blocks, reduce;
 };
 
@@ -65,6 +66,9 @@ struct CommitParams {
 
 specpv_status launch_summaries(const SummaryParams& p, int n_layers, int blocks_touched, int dtype, cudaStream_t stream);
 specpv_status launch_scores(const ScoreParams& p, int n_layers, int max_nb, int dtype, int d, cudaStream_t stream);
+bool scores_tc_supported(int dtype, int d, int G, int M_max);
+specpv_status launch_scores_tc(const ScoreParams& p, int n_layers_call, int n_layers_total, int max_nb,
+                               cudaStream_t stream);
 specpv_status launch_select(const SelectParams& p, int n_layers, cudaStream_t stream);
 specpv_status launch_gather(const GatherParams& p, int n_layers, cudaStream_t stream);
 specpv_status launch_commit(const CommitParams& p, int n_layers, int32_t* seq_lens, cudaStream_t stream);

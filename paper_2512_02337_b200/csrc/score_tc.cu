@@ -1,0 +1,248 @@
+// Block scores on the tensor cores (paper Eq. 2-3): s_i = f_r max(q_r . Kmax_i, q_r . Kmin_i) for
+// bfloat16 summaries with head_dim 128.
+//
+// Per (layer, sequence, KV head) the two products are dense contractions
+//     Dmax[128 blocks x R] = Kmax_tile[128 x 128] * Q^T[128 x R],   Dmin likewise with Kmin,
+// issued as tcgen05.mma with both operands in shared memory (128-byte swizzle, loaded by TMA) and
+// float32 accumulators in tensor memory (Dmax in columns [0, 256), Dmin in [256, 512)).  A CTA owns a
+// run of 128-block tiles of one head; thread i of the 128 epilogue threads owns block i of the tile
+// (tensor-memory lane i), takes max(Dmax, Dmin) per query row and reduces over the rows (mean, max,
+// or the rows of the "last" query).  The summaries of the next tile are in flight while a tile is
+// reduced.  Every wait is bounded.
+#include "aux_kernels.cuh"
+#include "tc_common.cuh"
+
+namespace specpv {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kScoreThreads = 192;       // warp 0: TMA + MMA issue, warp 1: idle, warps 2-5: epilogue (lane quarters 2,3,0,1)
+constexpr int kTileBlocks = 128;
+constexpr int kSumTileBytes = 32768;     // [2 d-halves][128 blocks][64 d] bf16
+constexpr int kScoreStages = 2;
+constexpr int kScoreQBytes = 65536;      // [2 d-halves][256 rows][64 d] bf16
+constexpr int kScoreSmem = 1024 + kScoreQBytes + kScoreStages * 2 * kSumTileBytes;
+
+struct ScoreTcParams {
+    CUtensorMap tm_q;     // (d, Hq, tokens)  box (64, G, 128/G)
+    CUtensorMap tm_kmax;  // (d, rows)        box (64, 128)
+    CUtensorMap tm_kmin;
+    const int32_t* q_lens;
+    const int32_t* last_query;
+    const int32_t* seq_lens;
+    float* scores;
+    void* workspace;
+    int layer0, batch, M_max, Hkv, G, bs, max_blocks, reduce, tiles_per_cta, n_cols;
+};
+
+struct __align__(8) ScoreBarriers {
+    uint64_t q_full;
+    uint64_t sum_full[kScoreStages];
+    uint64_t sum_empty[kScoreStages];
+    uint64_t d_full;
+    uint64_t d_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __grid_constant__ ScoreTcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ ScoreBarriers bars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, lb = blockIdx.z;
+    const int b = lb % p.batch, l = lb / p.batch;
+    const int seq_len = max(p.seq_lens[b], 0);
+    const int nb = min((seq_len + p.bs - 1) / p.bs, p.max_blocks);
+    const int tile_begin = blockIdx.x * p.tiles_per_cta;
+    const int tile_end = min(tile_begin + p.tiles_per_cta, (nb + kTileBlocks - 1) / kTileBlocks);
+    if (tile_begin >= tile_end) return;
+    const int n_tiles = tile_end - tile_begin;
+    int M = p.q_lens ? p.q_lens[b] : p.M_max;
+    M = min(max(M, 0), p.M_max);
+    int col_begin = 0, col_end = M * p.G;  // query rows r = token * G + head, one accumulator column each
+    if (p.reduce == SPECPV_REDUCE_LAST) {
+        int last = p.last_query ? p.last_query[b] : 0;
+        last = min(max(last, 0), max(M - 1, 0));
+        col_begin = last * p.G;
+        col_end = col_begin + p.G;
+    }
+    if (col_end <= col_begin) return;
+
+    const uint32_t q_smem = smem_u32(smem);
+    const uint32_t sum_smem = q_smem + kScoreQBytes;
+    volatile int* abort_flag = &bars.abort_flag;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars.q_full), 1);
+        for (int s = 0; s < kScoreStages; ++s) {
+            mbar_init(smem_u32(&bars.sum_full[s]), 1);
+            mbar_init(smem_u32(&bars.sum_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bars.d_full), 1);
+        mbar_init(smem_u32(&bars.d_empty), 128);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars.tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars.tmem_base;
+    const int tok_per_tile = 128 / p.G;
+    const uint32_t idesc = make_idesc((uint32_t)p.n_cols, false);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- producer + MMA issue (one thread) -------------------------------------------------
+            const uint32_t qbar = smem_u32(&bars.q_full);
+            const int n_q_tiles = p.n_cols > 128 ? 2 : 1;
+            mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
+            for (int t = 0; t < n_q_tiles; ++t)
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d(q_smem + half * 32768 + t * 16384, &p.tm_q, half * 64, h * p.G,
+                                lb * p.M_max + t * tok_per_tile, qbar);
+            const int row0 = (((p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks;
+            auto load_tile = [&](int i) {
+                const int slot = i % kScoreStages;
+                const uint32_t full = smem_u32(&bars.sum_full[slot]);
+                mbar_expect_tx(full, 2 * kSumTileBytes);
+                const uint32_t dst = sum_smem + slot * 2 * kSumTileBytes;
+                const int row = row0 + (tile_begin + i) * kTileBlocks;
+                for (int half = 0; half < 2; ++half) {
+                    tma_load_2d(dst + half * 16384, &p.tm_kmax, half * 64, row, full);
+                    tma_load_2d(dst + kSumTileBytes + half * 16384, &p.tm_kmin, half * 64, row, full);
+                }
+            };
+            load_tile(0);
+            bool ok = mbar_wait(qbar, 0, abort_flag, p.workspace, 20);
+            for (int i = 0; ok && i < n_tiles; ++i) {
+                if (i + 1 < n_tiles) {
+                    const int use = i + 1;
+                    if (use >= kScoreStages)
+                        ok = mbar_wait(smem_u32(&bars.sum_empty[use % kScoreStages]), ((use / kScoreStages) - 1) & 1,
+                                       abort_flag, p.workspace, 21);
+                    if (!ok) break;
+                    load_tile(use);
+                }
+                const int slot = i % kScoreStages;
+                ok = mbar_wait(smem_u32(&bars.sum_full[slot]), (i / kScoreStages) & 1, abort_flag, p.workspace, 22);
+                if (!ok) break;
+                if (i > 0) ok = mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_max = sum_smem + slot * 2 * kSumTileBytes, a_min = a_max + kSumTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t a_off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                    const uint32_t b_off = (kk >> 2) * 32768 + (kk & 3) * 32;
+                    const uint64_t bdesc = make_desc(q_smem + b_off, 16, 1024);
+                    mma_ss(tmem, make_desc(a_max + a_off, 16, 1024), bdesc, idesc, kk > 0);
+                    mma_ss(tmem + 256, make_desc(a_min + a_off, 16, 1024), bdesc, idesc, kk > 0);
+                }
+                tc_commit(smem_u32(&bars.d_full));
+                tc_commit(smem_u32(&bars.sum_empty[slot]));
+            }
+        }
+    } else if (warp >= 2) {
+        // ---- epilogue: thread <-> block of the tile -----------------------------------------------
+        const int q = warp & 3;  // tensor-memory lane quarter of this warp
+        const int blk_in_tile = q * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        bool ok = true;
+        for (int i = 0; i < n_tiles && ok; ++i) {
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full), i & 1, abort_flag, p.workspace, 24));
+            if (!ok) break;
+            tc_fence_after();
+            float red = p.reduce == SPECPV_REDUCE_MAX ? -INFINITY : 0.f;
+            for (int c0 = (col_begin / 32) * 32; c0 < col_end; c0 += 32) {
+                uint32_t vmax[32], vmin[32];
+                TMEM_LD32(tmem + lane_addr + c0, vmax);
+                TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
+                tmem_wait_ld();
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    const int c = c0 + k;
+                    const float s = fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
+                    if (c >= col_begin && c < col_end) red = p.reduce == SPECPV_REDUCE_MAX ? fmaxf(red, s) : red + s;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars.d_empty));
+            const int blk = (tile_begin + i) * kTileBlocks + blk_in_tile;
+            if (blk < nb) {
+                if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)(col_end - col_begin);
+                p.scores[((size_t)lb * p.Hkv + h) * p.max_blocks + blk] = red;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (*abort_flag) __nanosleep(200000);
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+}  // namespace
+
+bool scores_tc_supported(int dtype, int d, int G, int M_max) {
+    return dtype == SPECPV_DTYPE_BF16 && d == 128 && G <= 128 && (128 % G) == 0 && M_max * G <= 256 &&
+           tc::get_encode_fn() != nullptr;
+}
+
+specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_layers_total, int max_nb,
+                               cudaStream_t stream) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess)
+            return SPECPV_ERR_CUDA;
+        attr_set = true;
+    }
+    if (max_nb <= 0 || n_layers_call <= 0) return SPECPV_OK;
+    ScoreTcParams p{};
+    const uint64_t step_tokens = (uint64_t)n_layers_call * sp.batch * sp.M_max;
+    {
+        uint64_t dims[3] = {128, (uint64_t)sp.Hq, step_tokens};
+        uint64_t strides[2] = {256, (uint64_t)sp.Hq * 256};
+        uint32_t box[3] = {64, (uint32_t)sp.G, (uint32_t)(128 / sp.G)};
+        if (!tc::encode_map(&p.tm_q, sp.q, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
+    }
+    {
+        uint64_t dims[2] = {128, (uint64_t)n_layers_total * sp.batch * sp.Hkv * sp.max_blocks};
+        if (dims[1] >= 0x7FFFFF00ull) return SPECPV_ERR_UNSUPPORTED;
+        uint64_t strides[1] = {256};
+        uint32_t box[2] = {64, 128};
+        if (!tc::encode_map(&p.tm_kmax, sp.kmax, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
+        if (!tc::encode_map(&p.tm_kmin, sp.kmin, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
+    }
+    p.q_lens = sp.q_lens; p.last_query = sp.last_query; p.seq_lens = sp.seq_lens; p.scores = sp.scores;
+    p.workspace = sp.workspace;
+    p.layer0 = sp.layer0; p.batch = sp.batch; p.M_max = sp.M_max; p.Hkv = sp.Hkv; p.G = sp.G; p.bs = sp.bs;
+    p.max_blocks = sp.max_blocks; p.reduce = sp.reduce;
+    const int R = sp.M_max * sp.G;
+    p.n_cols = R <= 128 ? 128 : 256;  // accumulator columns = query rows, padded to whole 128-row Q tiles
+    const int n_tiles = (max_nb + kTileBlocks - 1) / kTileBlocks;
+    const int heads = sp.Hkv * n_layers_call * sp.batch;
+    // enough CTAs to fill the machine, but at least a few tiles each so that Q is amortised
+    int ctas_x = (2 * 148 + heads - 1) / heads;
+    if (ctas_x > n_tiles) ctas_x = n_tiles;
+    if (ctas_x < 1) ctas_x = 1;
+    p.tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
+    ctas_x = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
+    dim3 grid(ctas_x, sp.Hkv, n_layers_call * sp.batch);
+    scores_tc_kernel<<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+    count_launch();
+    return SPECPV_OK;
+}
+
+}  // namespace specpv

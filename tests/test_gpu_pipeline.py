@@ -118,6 +118,12 @@ def test_small_bf16_llama_shape_pipeline():
     run_pipeline("llama_32k", n_layers=2, ctx=[6144 + 37], M=60)
 
 
+@pytest.mark.parametrize("reduce", [1, 2])
+def test_small_bf16_other_reductions(reduce):
+    # max / last reductions through the tensor-core score kernel, M = 20 (80 query rows: one Q tile)
+    run_pipeline("llama_32k", n_layers=1, reduce=reduce, ctx=[64 * 150 + 11], M=20)
+
+
 def test_ragged_batch_shuffled_table_pipeline():
     run_pipeline("stress_b4", n_layers=1, ctx=[4096 + 5, 4800, 5120 - 1, 5120], M=64)
 
