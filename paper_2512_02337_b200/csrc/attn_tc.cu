@@ -57,6 +57,37 @@ struct TcParams {
 
 using namespace tc;
 
+// tcgen05.mma with the shared-memory descriptors given as (low word, common high word); `acc` = 0
+// overwrites D, anything else accumulates.
+__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                            uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                            uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// keeps the compiler from hoisting per-instruction descriptor words out of the tile loop
+__device__ __forceinline__ uint32_t launder(uint32_t x) {
+    asm volatile("" : "+r"(x));
+    return x;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128, N = 128.
 constexpr uint32_t kIdescQK = make_idesc(128, false);
 constexpr uint32_t kIdescPV = make_idesc(128, true);  // B (= V) is MN-major
@@ -66,8 +97,10 @@ struct __align__(8) Barriers {
     uint64_t kv_full[kStages];
     uint64_t kv_empty[kStages];
     uint64_t s_full[2];
-    uint64_t p_full[2];
+    uint64_t p_full[2][2];  // [row tile][half of the 128 tokens]
     uint64_t o_done[2];
+    uint64_t v_need;        // MMA issuer -> warp 2: this V tile has landed and needs its tail rows zeroed
+    uint64_t v_fixed;       // warp 2 -> MMA issuer: done
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -100,6 +133,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const bool last_split = split == p.n_splits - 1;
     const int n_ctx_tiles = tile_end - tile_begin;
     const int n_tiles = n_ctx_tiles + (last_split ? 1 : 0);  // the last split also attends the step's own tokens
+    // first tile whose V rows need zeroing past the valid tokens: a ragged last context tile, else the
+    // tile of the step's own tokens (fewer than 128), else none
+    const bool ragged_ctx = n_ctx_tiles > 0 && tile_end == total_tiles && (seq_len % kTileTokens) != 0;
+    const int first_fix = ragged_ctx ? n_ctx_tiles - 1 : ((last_split && M < kTileTokens) ? n_ctx_tiles : n_tiles);
 
     const uint32_t q_smem = smem_u32(smem);
     const uint32_t kv_smem = q_smem + kQBytes;
@@ -127,9 +164,12 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.p_full[t]), 128);
+            mbar_init(smem_u32(&bars.p_full[t][0]), 4);  // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.p_full[t][1]), 4);
             mbar_init(smem_u32(&bars.o_done[t]), 1);
         }
+        mbar_init(smem_u32(&bars.v_need), 1);
+        mbar_init(smem_u32(&bars.v_fixed), 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -158,22 +198,27 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                                 lb * p.M_max + tok0 + t * tok_per_tile, qbar);
             const int32_t* table = p.block_table + (size_t)b * p.max_blocks;
             const long long layer_row0 = (long long)(p.layer0 + l) * p.n_pages;
-            for (int j = 0; j < n_tiles; ++j) {
-                const bool is_new = j >= n_ctx_tiles;
-                int row[2];  // pool row coordinate of the tile's two pages
-                if (!is_new) {
-                    for (int pg = 0; pg < 2; ++pg) {
-                        const int blk = (tile_begin + j) * 2 + pg;
-                        row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
-                        if ((long long)blk * kPage < seq_len && blk < p.max_blocks) {
-                            const int page = table[blk];
-                            if (page < 0 || page >= p.n_pages)
-                                record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
-                            else
-                                row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
-                        }
+            // pool row coordinate of a context tile's two pages; the table is read one tile ahead so that
+            // its latency hides behind the wait for a free slot
+            auto page_rows = [&](int j, int* row) {
+                for (int pg = 0; pg < 2; ++pg) {
+                    const int blk = (tile_begin + j) * 2 + pg;
+                    row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
+                    if (j < n_ctx_tiles && (long long)blk * kPage < seq_len && blk < p.max_blocks) {
+                        const int page = table[blk];
+                        if (page < 0 || page >= p.n_pages)
+                            record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
+                        else
+                            row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
                     }
                 }
+            };
+            int row_next[2];
+            page_rows(0, row_next);
+            for (int j = 0; j < n_tiles; ++j) {
+                const bool is_new = j >= n_ctx_tiles;
+                const int row[2] = {row_next[0], row_next[1]};
+                page_rows(j + 1, row_next);
                 for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
                     const int use = 2 * j + kv;
                     const int slot = use % kStages;
@@ -196,33 +241,45 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     } else if (warp == 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== MMA issuer ==================================================
+        // The whole warp runs the loop (waits are warp-uniform); lane 0 issues.
         // Issue order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) | PV(0,1) QK(1,1) | ...
-        bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
+        // PV(j,t) is issued in two halves of 64 tokens, each as soon as the softmax warps have published
+        // that half of P, so that the first half runs while the second is still being exponentiated.
+        auto wait_all = [&](uint32_t bar, uint32_t parity, int where) {
+            return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.workspace, where));
+        };
+        bool ok = wait_all(smem_u32(&bars.q_full), 0, 2);
+        // Shared-memory descriptors: the upper word (stride between 8-row groups, version, swizzle) is
+        // constant; the lower word is the 16-byte address plus the leading-dimension offset.
+        const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
+        const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+        const uint32_t k_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+        const uint32_t v_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16384u >> 4) << 16);
         auto issue_qk = [&](int j, int t) {
-            const int slot = (2 * j) % kStages;
-            const uint32_t kbase = kv_smem + slot * kSlotBytes;
-            const uint32_t qbase = q_smem + t * 32768;
+            const uint32_t b_lo = launder(k_lo0 + (uint32_t)((2 * j) % kStages) * (kSlotBytes >> 4));
+            const uint32_t a_lo = launder(q_lo + (uint32_t)t * (32768u >> 4));
+            const uint32_t d = tmem + t * 128;
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
-                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                mma_ss(tmem + t * 128, make_desc(qbase + off, 16, 1024), make_desc(kbase + off, 16, 1024), kIdescQK,
-                       kk > 0);
+                const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                mma_ss_lohi(d, a_lo + off, b_lo + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
             }
         };
-        auto issue_pv = [&](int j, int t) {
-            const int slot = (2 * j + 1) % kStages;
-            const uint32_t vbase = kv_smem + slot * kSlotBytes;
+        auto issue_pv_half = [&](int j, int t, int half) {
+            const uint32_t b_lo = launder(v_lo0 + (uint32_t)((2 * j + 1) % kStages) * (kSlotBytes >> 4) +
+                                          (uint32_t)half * (4u * 2048u >> 4));
+            const uint32_t a = launder(tmem + t * 128 + half * 32);
+            const uint32_t d = tmem + 256 + t * 128;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
-                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, make_desc(vbase + kk * 2048, 16384, 1024),
-                       kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
-            }
+            for (int k4 = 0; k4 < 4; ++k4)  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
+                mma_ts_lohi(d, a + k4 * 8, b_lo + (uint32_t)k4 * (2048u >> 4), desc_hi, kIdescPV,
+                            (j > 0 || half > 0 || k4 > 0) ? 1u : 0u);
         };
         for (int j = 0; ok && j <= n_tiles; ++j) {
             if (j < n_tiles) {
                 // K tile of step j
                 const int use = 2 * j;
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, abort_flag, p.workspace, 3));
+                ok = wait_all(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, 3);
                 if (!ok) break;
                 tc_fence_after();
             }
@@ -232,33 +289,27 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     const int jp = j - 1;
                     if (t == 0) {
                         const int use = 2 * jp + 1;
-                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1,
-                                                                abort_flag, p.workspace, 4));
+                        ok = wait_all(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, 4);
                         if (!ok) break;
-                        // rows of V past the tile's valid tokens may hold anything: zero them so that
-                        // 0 * garbage cannot produce NaN
-                        const bool jp_new = jp >= n_ctx_tiles;
-                        const int n_valid = jp_new ? M : min(kTileTokens, seq_len - (tile_begin + jp) * kTileTokens);
-                        if (n_valid < kTileTokens) {
-                            uint8_t* v = smem + kQBytes + (size_t)(use % kStages) * kSlotBytes;
-                            const int n_rows = kTileTokens - n_valid;
-                            for (int i = lane; i < n_rows * 2 * 8; i += 32) {
-                                const int chunk = i & 7, half = (i >> 3) & 1, r = n_valid + (i >> 4);
-                                *reinterpret_cast<uint4*>(v + half * 16384 + r * 128 + chunk * 16) = make_uint4(0, 0, 0, 0);
-                            }
-                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                            __syncwarp();
+                        // a ragged or tree tile: warp 2 zeroes the rows of V past the valid tokens first
+                        if (jp >= first_fix) {
+                            if (lane == 0) mbar_arrive(smem_u32(&bars.v_need));
+                            ok = wait_all(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, 9);
+                            if (!ok) break;
                         }
                     }
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.p_full[t]), jp & 1, abort_flag, p.workspace, 5));
+                    for (int half = 0; half < 2 && ok; ++half) {
+                        ok = wait_all(smem_u32(&bars.p_full[t][half]), jp & 1, 5);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (lane == 0) issue_pv_half(jp, t, half);
+                        __syncwarp();
+                    }
                     if (!ok) break;
-                    tc_fence_after();
                     if (lane == 0) {
-                        issue_pv(jp, t);
                         tc_commit(smem_u32(&bars.o_done[t]));
                         if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.kv_empty[(2 * jp + 1) % kStages]));
                     }
-                    __syncwarp();
                 }
                 if (j < n_tiles) {
                     if (lane == 0) {
@@ -270,7 +321,30 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 }
             }
         }
-    } else if (warp < 4) {
+    } else if (warp == 2) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        // =========================== V fixer =====================================================
+        // Rows of a V tile past its valid tokens may hold anything (stale shared memory, rows of other
+        // sequences' steps): zero them so that 0 * garbage cannot produce NaN.  Only the last context
+        // tile (when ragged) and the tile of the step's own tokens can need it.
+        for (int jp = first_fix; jp < n_tiles; ++jp) {
+            const int use = 2 * jp + 1;
+            // the request arrives once the tile has landed (a wait on the slot's own barrier this far
+            // ahead of the pipeline could match an earlier phase of the same parity)
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_need), (jp - first_fix) & 1, abort_flag, p.workspace, 10)))
+                break;
+            const int n_valid = jp >= n_ctx_tiles ? M : min(kTileTokens, seq_len - (tile_begin + jp) * kTileTokens);
+            uint8_t* v = smem + kQBytes + (size_t)(use % kStages) * kSlotBytes;
+            const int n_rows = kTileTokens - n_valid;
+            for (int i = lane; i < n_rows * 2 * 8; i += 32) {
+                const int chunk = i & 7, half = (i >> 3) & 1, r = n_valid + (i >> 4);
+                *reinterpret_cast<uint4*>(v + half * 16384 + r * 128 + chunk * 16) = make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.v_fixed));
+        }
+    } else if (warp == 3) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
@@ -328,14 +402,17 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                         if (!((word >> (i & 63)) & 1ull)) v[i] = 0xff800000u;
                     }
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]), mx2 = __uint_as_float(v[2]),
+                      mx3 = __uint_as_float(v[3]);
 #pragma unroll
-                for (int i = 0; i < 128; i += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(v[i]));
-                    mx1 = fmaxf(mx1, __uint_as_float(v[i + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(v[i + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(v[i + 3]));
+                for (int i = 4; i < 124; i += 8) {  // three-input max: two new values per instruction
+                    mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
                 }
+                mx0 = fmax3(mx0, __uint_as_float(v[124]), __uint_as_float(v[125]));
+                mx1 = fmax3(mx1, __uint_as_float(v[126]), __uint_as_float(v[127]));
                 const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 const float m_tile = mx * p.scale_log2;
                 // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger.
@@ -383,14 +460,22 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
                     v[i] = w;
                     sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
-                    if (i == 31) TMEM_ST32(s_addr, v);
+                    if (i == 31) TMEM_ST32(s_addr, v);  // tokens 0..63 of P
+                    if (i == 39) {
+                        // the store above has had time to land: publish the first half so that its PV can start
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t][0]));
+                    }
                 }
                 TMEM_ST32(s_addr + 32, (v + 32));
                 const float l_add = sum2.x + sum2.y;
                 l_run += l_add;
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(smem_u32(&bars.p_full[t]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t][1]));
             }
             // ---- epilogue: wait for the last PV, normalise, write out ---------------------------
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), (n_tiles - 1) & 1, abort_flag, p.workspace, 8));
