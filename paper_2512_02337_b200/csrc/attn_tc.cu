@@ -94,13 +94,13 @@ constexpr uint32_t kIdescPV = make_idesc(128, true);  // B (= V) is MN-major
 
 struct __align__(8) Barriers {
     uint64_t q_full;
-    uint64_t kv_full[kStages];
-    uint64_t kv_empty[kStages];
-    uint64_t s_full[2];
-    uint64_t p_full[2][2];  // [row tile][half of the 128 tokens]
-    uint64_t o_done[2];
-    uint64_t v_need;        // MMA issuer -> warp 2: this V tile has landed and needs its tail rows zeroed
-    uint64_t v_fixed;       // warp 2 -> MMA issuer: done
+    uint64_t kv_full[kStages];  // a K or V tile has landed in its slot
+    uint64_t v_free;            // phase j: PV(j) of the last row tile has completed, V tile j's slot is free
+    uint64_t s_full[2];         // phase j: S_t(j) = Q_t K_j^T is complete (for the last row tile: K tile j's slot is free too)
+    uint64_t p_full[2];         // phase j: the four softmax warps of row tile t have stored P_t(j)
+    uint64_t o_done[2];         // the last PV of row tile t has completed
+    uint64_t v_need;            // MMA issuer -> warp 2: this V tile has landed and needs its tail rows zeroed
+    uint64_t v_fixed;           // warp 2 -> MMA issuer: done
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -158,14 +158,11 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     // ---- set-up ------------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars.q_full), 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bars.kv_full[s]), 1);
-            mbar_init(smem_u32(&bars.kv_empty[s]), 1);
-        }
+        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars.kv_full[s]), 1);
+        mbar_init(smem_u32(&bars.v_free), 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.p_full[t][0]), 4);  // one arrival per softmax warp
-            mbar_init(smem_u32(&bars.p_full[t][1]), 4);
+            mbar_init(smem_u32(&bars.p_full[t]), 4);  // one arrival per softmax warp
             mbar_init(smem_u32(&bars.o_done[t]), 1);
         }
         mbar_init(smem_u32(&bars.v_need), 1);
@@ -222,8 +219,14 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
                     const int use = 2 * j + kv;
                     const int slot = use % kStages;
-                    const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
-                    if (use >= kStages && !mbar_wait(empty, ((use / kStages) - 1) & 1, abort_flag, p.workspace, 1)) break;
+                    const uint32_t full = smem_u32(&bars.kv_full[slot]);
+                    if (use >= kStages) {
+                        // the slot's previous tenant: K tile j goes where V tile j-3 was (free once its PV is
+                        // done), V tile j where K tile j-2 was (free once S(j-2) of the last row tile is done)
+                        const int prev = kv ? j - 2 : j - 3;
+                        const uint32_t freed = kv ? smem_u32(&bars.s_full[n_q_tiles - 1]) : smem_u32(&bars.v_free);
+                        if (!mbar_wait(freed, prev & 1, abort_flag, p.workspace, 1)) break;
+                    }
                     mbar_expect_tx(full, kSlotBytes);
                     const uint32_t dst = kv_smem + slot * kSlotBytes;
                     for (int pg = 0; pg < 2; ++pg)
@@ -241,86 +244,68 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     } else if (warp == 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== MMA issuer ==================================================
-        // The whole warp runs the loop (waits are warp-uniform); lane 0 issues.
-        // Issue order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) | PV(0,1) QK(1,1) | ...
-        // PV(j,t) is issued in two halves of 64 tokens, each as soon as the softmax warps have published
-        // that half of P, so that the first half runs while the second is still being exponentiated.
-        auto wait_all = [&](uint32_t bar, uint32_t parity, int where) {
-            return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.workspace, where));
-        };
-        bool ok = wait_all(smem_u32(&bars.q_full), 0, 2);
+        // One warp issues every contraction (issuing from two warps serialises the tensor pipe).  Issue
+        // order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | ...
+        // Barrier instructions do not overlap with queued MMAs (each costs the pipe 30-100 idle cycles),
+        // so the loop keeps them to four waits per KV tile, without votes, and three commits, each right
+        // behind eight MMAs.  The whole warp runs the loop, lane 0 issues.  A wait that gives up makes
+        // every later wait return at once (abort flag), so the loop simply runs out.
+        bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
         // Shared-memory descriptors: the upper word (stride between 8-row groups, version, swizzle) is
         // constant; the lower word is the 16-byte address plus the leading-dimension offset.
         const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
         const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
         const uint32_t k_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
         const uint32_t v_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16384u >> 4) << 16);
-        auto issue_qk = [&](int j, int t) {
-            const uint32_t b_lo = launder(k_lo0 + (uint32_t)((2 * j) % kStages) * (kSlotBytes >> 4));
-            const uint32_t a_lo = launder(q_lo + (uint32_t)t * (32768u >> 4));
-            const uint32_t d = tmem + t * 128;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
-                const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
-                mma_ss_lohi(d, a_lo + off, b_lo + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
+        const uint32_t full0 = smem_u32(&bars.kv_full[0]);
+        const uint32_t sfull0 = smem_u32(&bars.s_full[0]), pfull0 = smem_u32(&bars.p_full[0]);
+        // ring position of K tile j (use 2j) and of V tile j-1 (use 2j-1): slot and phase parity
+        uint32_t k_slot = 0, k_par = 0, v_slot = 1, v_par = 0;
+        for (int j = 0; j <= n_tiles; ++j) {
+            const int jp = j - 1;
+            if (j < n_tiles) ok &= mbar_wait(full0 + k_slot * 8, k_par, abort_flag, p.workspace, 3);
+            if (j > 0) {
+                ok &= mbar_wait(full0 + v_slot * 8, v_par, abort_flag, p.workspace, 4);
+                // a ragged or tree tile: warp 2 zeroes the rows of V past the valid tokens first
+                if (jp >= first_fix) {
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.v_need));
+                    ok &= mbar_wait(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, abort_flag, p.workspace, 9);
+                }
             }
-        };
-        auto issue_pv_half = [&](int j, int t, int half) {
-            const uint32_t b_lo = launder(v_lo0 + (uint32_t)((2 * j + 1) % kStages) * (kSlotBytes >> 4) +
-                                          (uint32_t)half * (4u * 2048u >> 4));
-            const uint32_t a = launder(tmem + t * 128 + half * 32);
-            const uint32_t d = tmem + 256 + t * 128;
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
-                mma_ts_lohi(d, a + k4 * 8, b_lo + (uint32_t)k4 * (2048u >> 4), desc_hi, kIdescPV,
-                            (j > 0 || half > 0 || k4 > 0) ? 1u : 0u);
-        };
-        for (int j = 0; ok && j <= n_tiles; ++j) {
-            if (j < n_tiles) {
-                // K tile of step j
-                const int use = 2 * j;
-                ok = wait_all(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, 3);
-                if (!ok) break;
-                tc_fence_after();
-            }
-            for (int t = 0; t < n_q_tiles && ok; ++t) {
+            const uint32_t kb_lo = launder(k_lo0 + k_slot * (kSlotBytes >> 4));
+            const uint32_t vb_lo = launder(v_lo0 + v_slot * (kSlotBytes >> 4));
+            for (int t = 0; t < n_q_tiles; ++t) {
                 if (j > 0) {
-                    // PV of the previous tile for this row tile
-                    const int jp = j - 1;
-                    if (t == 0) {
-                        const int use = 2 * jp + 1;
-                        ok = wait_all(smem_u32(&bars.kv_full[use % kStages]), (use / kStages) & 1, 4);
-                        if (!ok) break;
-                        // a ragged or tree tile: warp 2 zeroes the rows of V past the valid tokens first
-                        if (jp >= first_fix) {
-                            if (lane == 0) mbar_arrive(smem_u32(&bars.v_need));
-                            ok = wait_all(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, 9);
-                            if (!ok) break;
+                    ok &= mbar_wait(pfull0 + t * 8, jp & 1, abort_flag, p.workspace, 5);
+                    tc_fence_after();
+                }
+                if (lane == 0) {
+                    if (j > 0) {  // O_t += P_t V_{j-1}
+                        const uint32_t a = tmem + t * 128, d = tmem + 256 + t * 128;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
+                            mma_ts_lohi(d, a + kk * 8, vb_lo + (uint32_t)kk * (2048u >> 4), desc_hi, kIdescPV,
+                                        (jp > 0 || kk > 0) ? 1u : 0u);
+                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.v_free));
+                        if (j == n_tiles) tc_commit(smem_u32(&bars.o_done[t]));
+                    }
+                    if (j < n_tiles) {  // S_t = Q_t K_j^T
+                        const uint32_t a_lo = launder(q_lo + (uint32_t)t * (32768u >> 4));
+                        const uint32_t d = tmem + t * 128;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
+                            const uint32_t off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                            mma_ss_lohi(d, a_lo + off, kb_lo + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
                         }
-                    }
-                    for (int half = 0; half < 2 && ok; ++half) {
-                        ok = wait_all(smem_u32(&bars.p_full[t][half]), jp & 1, 5);
-                        if (!ok) break;
-                        tc_fence_after();
-                        if (lane == 0) issue_pv_half(jp, t, half);
-                        __syncwarp();
-                    }
-                    if (!ok) break;
-                    if (lane == 0) {
-                        tc_commit(smem_u32(&bars.o_done[t]));
-                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.kv_empty[(2 * jp + 1) % kStages]));
+                        tc_commit(sfull0 + t * 8);
                     }
                 }
-                if (j < n_tiles) {
-                    if (lane == 0) {
-                        issue_qk(j, t);
-                        tc_commit(smem_u32(&bars.s_full[t]));
-                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.kv_empty[(2 * j) % kStages]));
-                    }
-                    __syncwarp();
-                }
+                __syncwarp();
             }
+            if (j < n_tiles) { k_slot += 2; if (k_slot >= kStages) { k_slot -= kStages; k_par ^= 1; } }
+            if (j > 0) { v_slot += 2; if (v_slot >= kStages) { v_slot -= kStages; v_par ^= 1; } }
         }
+        (void)ok;
     } else if (warp == 2) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== V fixer =====================================================
@@ -426,10 +411,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 }
                 if (__any_sync(0xffffffffu, need)) {
                     const float factor = !need ? 1.f : (m_run == -INFINITY ? 0.f : ex2(m_run - m_tile));
-                    // O_t must hold every earlier PV before it is rescaled
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag, p.workspace, 7));
-                    if (!ok) break;
-                    tc_fence_after();
+                    // O_t already holds every earlier PV: the tensor pipe runs in order, and S_t(j), issued
+                    // after PV(j-1,t), is complete
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t o[32];
@@ -461,13 +444,6 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     v[i] = w;
                     sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
                     if (i == 31) TMEM_ST32(s_addr, v);  // tokens 0..63 of P
-                    if (i == 39) {
-                        // the store above has had time to land: publish the first half so that its PV can start
-                        tmem_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t][0]));
-                    }
                 }
                 TMEM_ST32(s_addr + 32, (v + 32));
                 const float l_add = sum2.x + sum2.y;
@@ -475,10 +451,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t][1]));
+                if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
             }
             // ---- epilogue: wait for the last PV, normalise, write out ---------------------------
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), (n_tiles - 1) & 1, abort_flag, p.workspace, 8));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_done[t]), 0, abort_flag, p.workspace, 8));
             if (ok) {
                 tc_fence_after();
                 const bool direct = p.n_splits == 1;
