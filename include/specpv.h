@@ -179,6 +179,40 @@ specpv_status specpv_verify_full(const specpv_config *cfg, int layer0, int n_lay
                                  void *out, float *lse, void *workspace, size_t workspace_bytes,
                                  void *stream);
 
+/* (No counterpart in the paper: an allocation-free variant of specpv_verify_partial.)
+ *
+ * Some callers cannot give this library a workspace because they cannot allocate device memory at
+ * the point where they call it: an inference server that handed all of the GPU's memory to its own
+ * KV-cache pool at start-up, a plug-in that runs inside such a server's decode loop where a
+ * cudaMalloc would stall every stream of the device (or simply fail because nothing is left), or a
+ * process whose allocator is owned by another component.  For them this call keeps its split-KV
+ * scratch and its status word in a fixed array of SPECPV_STATIC_SCRATCH_BYTES that is part of the
+ * library image: every GPU on which the library is used holds that array from the first use until
+ * the process exits, whether or not this call is ever made again.  The call itself performs no
+ * cudaMalloc / cudaFree and calls no allocating routine; q, k_new, v_new, tree_mask, the partial
+ * cache, out and lse are still the caller's device buffers, with the meaning they have in
+ * specpv_verify_partial.
+ *
+ * Limit: n_layers * batch * Hkv * ceil(M_max * G / 256) * 256 * (head_dim + 2) * 4 bytes (one
+ * KV split's partial results) must fit twice into SPECPV_STATIC_SCRATCH_BYTES - 256; a larger
+ * request returns SPECPV_ERR_CAPACITY and launches nothing.  Within the limit the scratch only
+ * bounds how many KV splits are used, never the result.
+ *
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  Every call uses the same array: two calls
+ * whose kernels can overlap on the GPU (different streams without an ordering between them) race
+ * on it; calls on one stream, or ordered by events, are safe.  The array keeps the previous
+ * call's partial results; nothing in it needs to start at zero except the status word, which the
+ * call clears on `stream` before launching.  device_status (device, 5 x int32, nullable) receives
+ * a copy of the status word at the end of the call's work on `stream`: word 0 is the first
+ * device-detected specpv_status of this call (0 = none), words 1..4 its details. */
+#define SPECPV_STATIC_SCRATCH_BYTES (16u << 20)
+specpv_status specpv_verify_partial_static(const specpv_config *cfg, int layer0, int n_layers,
+                                           const void *q, const void *k_new, const void *v_new,
+                                           const uint64_t *tree_mask, const int32_t *q_lens, int M_max,
+                                           const specpv_paged_kv *partial, void *out, float *lse,
+                                           int32_t *device_status, void *stream);
+
 /* The same step with HOST step tensors (q, k_new, v_new, tree_mask, out, lse are host pointers,
  * ideally pinned): copies the inputs to staging space inside the workspace, runs the attention
  * (mode = SPECPV_MODE_PARTIAL or SPECPV_MODE_FULL selects only validation), copies out/lse back and

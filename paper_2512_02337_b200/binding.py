@@ -26,7 +26,7 @@ EXPORTS = [
     "specpv_status_string", "specpv_workspace_bytes", "specpv_kernel_launches", "specpv_poll_status", "specpv_build_tree_mask",
     "specpv_select_mode", "specpv_update_block_summaries", "specpv_score_blocks",
     "specpv_select_partial_kv", "specpv_refresh_partial", "specpv_verify_partial",
-    "specpv_verify_full", "specpv_verify_host", "specpv_commit_accepted",
+    "specpv_verify_full", "specpv_verify_host", "specpv_commit_accepted", "specpv_verify_partial_static",
 ]
 
 
@@ -207,6 +207,21 @@ def specpv_verify_partial(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_l
                           lse, workspace, stream=None):
     _verify("specpv_verify_partial", cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, partial,
             out, lse, workspace, stream)
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def specpv_verify_partial_static(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, partial: Cache,
+                                 out, lse, device_status=None, stream=None):
+    """specpv_verify_partial without a workspace: the scratch is a fixed array inside the library, so the
+    call allocates nothing (for callers whose device memory is all spoken for).  ``device_status`` is an
+    optional int32 device tensor of 5 words that receives the call's device-side status."""
+    d = partial.desc()
+    _check(lib().specpv_verify_partial_static(ctypes.byref(cfg), layer0, n_layers, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                              _ptr(tree_mask), _ptr(q_lens), M_max, ctypes.byref(d), _ptr(out),
+                                              _ptr(lse), _ptr(device_status), _stream(stream)),
+           "specpv_verify_partial_static")
 
 
 def specpv_verify_full(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, full: Cache, out, lse,

@@ -10,6 +10,7 @@
 #define SPECPV_EXPORT extern "C" __attribute__((visibility("default")))
 
 #include <atomic>
+#include <mutex>
 
 namespace specpv {
 
@@ -289,6 +290,79 @@ SPECPV_EXPORT specpv_status specpv_verify_partial(const specpv_config* cfg, int 
                                                   void* stream) {
     return verify_common(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, partial, out, lse,
                          workspace, workspace_bytes, stream, true);
+}
+
+// ---- allocation-free variant of specpv_verify_partial -------------------------------------------
+// The scratch lives in the library image.  In host code the array's name is only a handle for the
+// runtime, not a device address: the address is looked up once per device and that is what the
+// kernels get.
+static __device__ __align__(256) unsigned char g_static_scratch[SPECPV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_addr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up on first use).
+specpv_status static_scratch(void** addr) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPECPV_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return SPECPV_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return SPECPV_ERR_CUDA;
+        g_static_addr[dev] = ptr;
+    }
+    *addr = g_static_addr[dev];
+    return SPECPV_OK;
+}
+}  // namespace
+
+SPECPV_EXPORT specpv_status specpv_verify_partial_static(const specpv_config* cfg, int layer0, int n_layers,
+                                                         const void* q, const void* k_new, const void* v_new,
+                                                         const uint64_t* tree_mask, const int32_t* q_lens, int M_max,
+                                                         const specpv_paged_kv* partial, void* out, float* lse,
+                                                         int32_t* device_status, void* stream) {
+    Geometry g;
+    specpv_status st = validate_config(cfg, &g);
+    if (st != SPECPV_OK) return st;
+    st = validate_kv(g, partial);
+    if (st != SPECPV_OK) return st;
+    if (!q || !k_new || !v_new || !tree_mask || !out) return SPECPV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return SPECPV_ERR_INVALID_ARG;
+    if (layer0 < 0 || n_layers <= 0 || layer0 + n_layers > g.n_layers || M_max <= 0) return SPECPV_ERR_INVALID_ARG;
+    if (M_max > kMaxQTokens) return SPECPV_ERR_CAPACITY;
+    if ((int64_t)partial->max_blocks * g.bs < (int64_t)g.budget_blocks * g.bs + g.buffer_tokens) return SPECPV_ERR_CAPACITY;
+    // the fixed scratch must hold the partial results of at least two KV splits
+    const size_t scratch = (size_t)SPECPV_STATIC_SCRATCH_BYTES - kStatusBytes;
+    const size_t per_split = (size_t)n_layers * partial->batch * g.Hkv * round_up((size_t)M_max * g.G, 256) *
+                             (g.d + 2) * sizeof(float);
+    if (per_split > scratch / 2) return SPECPV_ERR_CAPACITY;
+    void* base = nullptr;
+    st = static_scratch(&base);
+    if (st != SPECPV_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // the status word is the only part of the array that has to start at zero
+    if (cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return SPECPV_ERR_CUDA;
+
+    AttnArgs a{};
+    a.g = g;
+    a.layer0 = layer0; a.n_layers = n_layers; a.batch = partial->batch; a.M_max = M_max;
+    a.mask_words = (M_max + 63) / 64;
+    a.q = q; a.k_new = k_new; a.v_new = v_new; a.tree_mask = tree_mask; a.q_lens = q_lens;
+    a.k_pool = partial->k_pool; a.v_pool = partial->v_pool; a.block_table = partial->block_table;
+    a.seq_lens = partial->seq_lens;
+    a.max_blocks = partial->max_blocks; a.n_pages = partial->n_pages; a.max_seq_len = partial->max_seq_len;
+    a.out = out; a.lse = lse; a.workspace = base;
+    a.partial_off = kStatusBytes;
+    a.partial_bytes = scratch;
+    st = attention_tc_supported(a) ? launch_attention_tc(a, s) : launch_attention_simt(a, s);
+    if (st != SPECPV_OK) return st;
+    if (device_status &&
+        cudaMemcpyAsync(device_status, base, sizeof(StatusWord), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return SPECPV_ERR_CUDA;
+    return SPECPV_OK;
 }
 
 SPECPV_EXPORT specpv_status specpv_verify_full(const specpv_config* cfg, int layer0, int n_layers, const void* q,
