@@ -33,6 +33,7 @@ constexpr int kSmemBytes = 1024 + kQBytes + kStages * kSlotBytes;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kSafeRowSum = 1.1529215e18f;  // 2^60: a tile's row sum below this cannot overflow the float32 sums
 
 struct TcParams {
     CUtensorMap tm_q;      // (d, Hq, tokens)          box (64, G, 128/G)
@@ -353,6 +354,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             }
             float m_run = -INFINITY, l_run = 0.f;
             bool ok = true;
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const bool is_new = j >= n_ctx_tiles;
                 const int n_valid = is_new ? M : min(kTileTokens, seq_len - (tile_begin + j) * kTileTokens);
@@ -380,73 +382,95 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 TMEM_LD32(s_addr + 64, (v + 64));
                 TMEM_LD32(s_addr + 96, (v + 96));
                 tmem_wait_ld();
-                if (masked) {  // ragged or tree-masked tile: invisible columns become -inf (at most two tiles per CTA)
+                // P = 2^(s*scale - m) as bf16 pairs, packed in place: word i of P (columns 2i, 2i+1) overwrites
+                // v[i], whose own value was consumed by an earlier pair, so no second register array is needed.
+                // The row sum is taken over the ROUNDED weights the tensor core will use, so that O / l is an
+                // exact weighted average of V rows (the rounding error of a dominant weight cancels instead of
+                // scaling the output).
+                auto exp_row = [&](float m_use) {
+                    const float2 nm2 = make_float2(-m_use, -m_use);
+                    float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) {
-                        const uint64_t word = i < 64 ? vis_lo : vis_hi;
-                        if (!((word >> (i & 63)) & 1ull)) v[i] = 0xff800000u;
+                    for (int i = 0; i < 64; ++i) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])),
+                                                    sc2, nm2);
+                        const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
+                        v[i] = w;
+                        sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
                     }
-                }
-                float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]), mx2 = __uint_as_float(v[2]),
-                      mx3 = __uint_as_float(v[3]);
-#pragma unroll
-                for (int i = 4; i < 124; i += 8) {  // three-input max: two new values per instruction
-                    mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-                    mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                    mx2 = fmax3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-                    mx3 = fmax3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-                }
-                mx0 = fmax3(mx0, __uint_as_float(v[124]), __uint_as_float(v[125]));
-                mx1 = fmax3(mx1, __uint_as_float(v[126]), __uint_as_float(v[127]));
-                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                const float m_tile = mx * p.scale_log2;
-                // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger.
-                // The decision is per row, the tensor-memory traffic is warp-wide: if any row of the
-                // warp rescales, all 32 rows pass through it (with a factor of 1 where nothing changes).
-                bool need = false;
-                if (j == 0) {
-                    m_run = m_tile;
-                } else {
-                    need = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
-                }
-                if (__any_sync(0xffffffffu, need)) {
-                    const float factor = !need ? 1.f : (m_run == -INFINITY ? 0.f : ex2(m_run - m_tile));
-                    // O_t already holds every earlier PV: the tensor pipe runs in order, and S_t(j), issued
-                    // after PV(j-1,t), is complete
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        TMEM_LD32(o_addr + c * 32, o);
+                    return sum2.x + sum2.y;
+                };
+                // Fast path (every full context tile after the first): keep the reference m_run of the row as it
+                // is and skip the row maximum.  Weights may then exceed 1; float32 sums and bf16 weights keep
+                // their relative precision whatever the exponent, so only overflow has to be ruled out: if a
+                // row sum leaves the safe range (or a row has no reference yet), the warp takes the tile again
+                // from tensor memory on the general path, which brings m_run up to date.
+                float l_add = 0.f;
+                bool general = j == 0 || masked;
+                if (!general) {
+                    l_add = exp_row(m_run);
+                    const bool bad = !(l_add < kSafeRowSum) || m_run == -INFINITY;
+                    if (__any_sync(0xffffffffu, bad)) {
+                        general = true;  // S_t is still intact: P has not been stored yet
+                        TMEM_LD32(s_addr, v);
+                        TMEM_LD32(s_addr + 32, (v + 32));
+                        TMEM_LD32(s_addr + 64, (v + 64));
+                        TMEM_LD32(s_addr + 96, (v + 96));
                         tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                        TMEM_ST32(o_addr + c * 32, o);
                     }
-                    if (need) {
-                        l_run *= factor;
+                }
+                if (general) {
+                    if (masked) {  // ragged or tree-masked tile: invisible columns become -inf (at most two tiles per CTA)
+#pragma unroll
+                        for (int i = 0; i < 128; ++i) {
+                            const uint64_t word = i < 64 ? vis_lo : vis_hi;
+                            if (!((word >> (i & 63)) & 1ull)) v[i] = 0xff800000u;
+                        }
+                    }
+                    float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]), mx2 = __uint_as_float(v[2]),
+                          mx3 = __uint_as_float(v[3]);
+#pragma unroll
+                    for (int i = 4; i < 124; i += 8) {  // three-input max: two new values per instruction
+                        mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                        mx2 = fmax3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                        mx3 = fmax3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+                    }
+                    mx0 = fmax3(mx0, __uint_as_float(v[124]), __uint_as_float(v[125]));
+                    mx1 = fmax3(mx1, __uint_as_float(v[126]), __uint_as_float(v[127]));
+                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    const float m_tile = mx * p.scale_log2;
+                    // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger.
+                    // The decision is per row, the tensor-memory traffic is warp-wide: if any row of the
+                    // warp rescales, all 32 rows pass through it (with a factor of 1 where nothing changes).
+                    bool need = false;
+                    if (j == 0) {
                         m_run = m_tile;
+                    } else {
+                        need = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
                     }
-                }
-                const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-                // P = 2^(s*scale - m) as bf16 pairs written over S (all of S is already in registers).  The row sum is taken over the ROUNDED weights the
-                // tensor core will use, so that O / l is an exact weighted average of V rows (the rounding
-                // error of a dominant weight cancels instead of scaling the output).
-                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-                const float2 nm2 = make_float2(-m_use, -m_use);
-                float2 sum2 = make_float2(0.f, 0.f);
-                // packed in place: word i of P (columns 2i, 2i+1) overwrites v[i], whose own value was
-                // consumed by an earlier pair, so no second register array is needed
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float factor = !need ? 1.f : (m_run == -INFINITY ? 0.f : ex2(m_run - m_tile));
+                        // O_t already holds every earlier PV: the tensor pipe runs in order, and S_t(j), issued
+                        // after PV(j-1,t), is complete
 #pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])),
-                                                sc2, nm2);
-                    const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
-                    v[i] = w;
-                    sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
-                    if (i == 31) TMEM_ST32(s_addr, v);  // tokens 0..63 of P
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            TMEM_LD32(o_addr + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                            TMEM_ST32(o_addr + c * 32, o);
+                        }
+                        if (need) {
+                            l_run *= factor;
+                            m_run = m_tile;
+                        }
+                    }
+                    l_add = exp_row((m_run == -INFINITY) ? 0.f : m_run);
                 }
+                TMEM_ST32(s_addr, v);
                 TMEM_ST32(s_addr + 32, (v + 32));
-                const float l_add = sum2.x + sum2.y;
                 l_run += l_add;
                 tmem_wait_st();
                 tc_fence_before();
