@@ -96,8 +96,10 @@ constexpr uint32_t kIdescPV = make_idesc(128, true);  // B (= V) is MN-major
 struct __align__(8) Barriers {
     uint64_t q_full;
     uint64_t kv_full[kStages];  // a K or V tile has landed in its slot
-    uint64_t v_free;            // phase j: PV(j) of the last row tile has completed, V tile j's slot is free
-    uint64_t s_full[2];         // phase j: S_t(j) = Q_t K_j^T is complete (for the last row tile: K tile j's slot is free too)
+    uint64_t kv_empty[kStages]; // every contraction that reads the slot has completed (one barrier per slot: a barrier
+                                // shared by all slots could run two phases ahead of the producer, which a parity
+                                // wait cannot tell from none)
+    uint64_t s_full[2];         // phase j: S_t(j) = Q_t K_j^T is complete
     uint64_t p_full[2];         // phase j: the four softmax warps of row tile t have stored P_t(j)
     uint64_t o_done[2];         // the last PV of row tile t has completed
     uint64_t v_need;            // MMA issuer -> warp 2: this V tile has landed and needs its tail rows zeroed
@@ -159,8 +161,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     // ---- set-up ------------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars.q_full), 1);
-        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars.kv_full[s]), 1);
-        mbar_init(smem_u32(&bars.v_free), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bars.kv_full[s]), 1);
+            mbar_init(smem_u32(&bars.kv_empty[s]), 1);
+        }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
             mbar_init(smem_u32(&bars.p_full[t]), 4);  // one arrival per softmax warp
@@ -220,14 +224,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
                     const int use = 2 * j + kv;
                     const int slot = use % kStages;
-                    const uint32_t full = smem_u32(&bars.kv_full[slot]);
-                    if (use >= kStages) {
-                        // the slot's previous tenant: K tile j goes where V tile j-3 was (free once its PV is
-                        // done), V tile j where K tile j-2 was (free once S(j-2) of the last row tile is done)
-                        const int prev = kv ? j - 2 : j - 3;
-                        const uint32_t freed = kv ? smem_u32(&bars.s_full[n_q_tiles - 1]) : smem_u32(&bars.v_free);
-                        if (!mbar_wait(freed, prev & 1, abort_flag, p.workspace, 1)) break;
-                    }
+                    const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
+                    if (use >= kStages && !mbar_wait(empty, ((use / kStages) - 1) & 1, abort_flag, p.workspace, 1)) break;
                     mbar_expect_tx(full, kSlotBytes);
                     const uint32_t dst = kv_smem + slot * kSlotBytes;
                     for (int pg = 0; pg < 2; ++pg)
@@ -248,8 +246,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         // One warp issues every contraction (issuing from two warps serialises the tensor pipe).  Issue
         // order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | ...
         // Barrier instructions do not overlap with queued MMAs (each costs the pipe 30-100 idle cycles),
-        // so the loop keeps them to four waits per KV tile, without votes, and three commits, each right
-        // behind eight MMAs.  The whole warp runs the loop, lane 0 issues.  A wait that gives up makes
+        // so the loop keeps them to four waits per KV tile, without votes, and four commits behind MMAs.  The whole warp runs the loop, lane 0 issues.  A wait that gives up makes
         // every later wait return at once (abort flag), so the loop simply runs out.
         bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
         // Shared-memory descriptors: the upper word (stride between 8-row groups, version, swizzle) is
@@ -258,7 +255,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
         const uint32_t k_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
         const uint32_t v_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16384u >> 4) << 16);
-        const uint32_t full0 = smem_u32(&bars.kv_full[0]);
+        const uint32_t full0 = smem_u32(&bars.kv_full[0]), empty0 = smem_u32(&bars.kv_empty[0]);
         const uint32_t sfull0 = smem_u32(&bars.s_full[0]), pfull0 = smem_u32(&bars.p_full[0]);
         // ring position of K tile j (use 2j) and of V tile j-1 (use 2j-1): slot and phase parity
         uint32_t k_slot = 0, k_par = 0, v_slot = 1, v_par = 0;
@@ -287,7 +284,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                         for (int kk = 0; kk < 8; ++kk)  // 16 tokens per instruction: two 8-row K groups of 1024 bytes
                             mma_ts_lohi(d, a + kk * 8, vb_lo + (uint32_t)kk * (2048u >> 4), desc_hi, kIdescPV,
                                         (jp > 0 || kk > 0) ? 1u : 0u);
-                        if (t == n_q_tiles - 1) tc_commit(smem_u32(&bars.v_free));
+                        if (t == n_q_tiles - 1) tc_commit(empty0 + v_slot * 8);
                         if (j == n_tiles) tc_commit(smem_u32(&bars.o_done[t]));
                     }
                     if (j < n_tiles) {  // S_t = Q_t K_j^T
@@ -299,6 +296,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                             mma_ss_lohi(d, a_lo + off, kb_lo + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
                         }
                         tc_commit(sfull0 + t * 8);
+                        if (t == n_q_tiles - 1) tc_commit(empty0 + k_slot * 8);
                     }
                 }
                 __syncwarp();
