@@ -58,7 +58,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -67,9 +67,10 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
 
-    def stop(self) -> dict:
+    def stop(self, t_begin: float = 0.0, t_end: float = float("inf")) -> dict:
+        """Summary of the samples that arrived inside [t_begin, t_end] (host clock of the timed region)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -78,19 +79,22 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for t, r in self.rows:
+            if not (t_begin <= t <= t_end + 0.03):
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                power.append(float(r[2]))
             except (ValueError, IndexError):
                 continue
             for name, val in zip(names, r[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "power_w": statistics.median(power) if power else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
 def build_state(name: str, device, n_layers=None, budget_blocks=None):
@@ -202,11 +206,13 @@ def timed_loop(st, steps, warmup, e2e, dist_barrier):
     torch.cuda.synchronize(dev)
     dist_barrier()
     launches0 = st["B"].specpv_kernel_launches()
+    wall0 = time.time()
     t0.record()
     for i in range(steps):
         run_step(st, e2e, ev[i])
     t1.record()
     torch.cuda.synchronize(dev)
+    wall1 = time.time()
     dist_barrier()
     total_ms = t0.elapsed_time(t1)
     full_ms = [e[0].elapsed_time(e[1]) for e in ev]
@@ -214,7 +220,7 @@ def timed_loop(st, steps, warmup, e2e, dist_barrier):
     st_code, info = st["B"].specpv_poll_status(st["ws"])
     if st_code != 0:
         raise RuntimeError(f"device status {st_code} {info}")
-    return total_ms / steps, full_ms, part_ms, st["B"].specpv_kernel_launches() - launches0
+    return total_ms / steps, full_ms, part_ms, st["B"].specpv_kernel_launches() - launches0, (wall0, wall1)
 
 
 def algorithmic_work(st):
@@ -266,7 +272,7 @@ def oracle_sample(st, budget_s=20.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama_128k", choices=list(wl.CONFIGS))
@@ -305,11 +311,12 @@ def main():
     c = st["w"].cfg
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
     sampler.start()
-    ms_step, full_ms, part_ms, launches = timed_loop(st, args.steps, warmup, False, barrier)
-    clocks = sampler.stop()
+    time.sleep(0.3)  # let the sampler deliver its first rows before the warm-up starts
+    ms_step, full_ms, part_ms, launches, window = timed_loop(st, args.steps, warmup, False, barrier)
+    clocks = sampler.stop(*window)
     e2e = None
     if not args.no_e2e:
-        e2e_ms, _, _, _ = timed_loop(st, args.steps, warmup, True, barrier)
+        e2e_ms, _, _, _, _ = timed_loop(st, args.steps, warmup, True, barrier)
     if use_dist:
         import torch.distributed as dist
         t = torch.tensor([ms_step, e2e_ms if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)

@@ -534,31 +534,47 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     }
 }
 
-// Log-sum-exp merge of the KV splits: grid = (R rows, Hkv, layers x seqs), one thread per channel.
-__global__ void __launch_bounds__(kD) merge_tc_kernel(TcParams p) {
-    const int r = blockIdx.x, h = blockIdx.y, lb = blockIdx.z, c = threadIdx.x;
+// Log-sum-exp merge of the KV splits: one warp per output row (a thread owns four channels), eight rows per
+// CTA; grid = (row groups, Hkv, layers x seqs).
+constexpr int kMergeRows = 8;
+__global__ void __launch_bounds__(32 * kMergeRows) merge_tc_kernel(TcParams p) {
+    const int r = blockIdx.x * kMergeRows + (threadIdx.x >> 5), h = blockIdx.y, lb = blockIdx.z, lane = threadIdx.x & 31;
     const int b = lb % p.batch;
     int M = p.q_lens ? p.q_lens[b] : p.M_max;
     M = min(max(M, 0), p.M_max);
     if (r >= M * p.G) return;
     const size_t base = ((size_t)lb * p.Hkv + h) * p.n_splits;
+    const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
     float m_all = -INFINITY;
-    for (int s = 0; s < p.n_splits; ++s) m_all = fmaxf(m_all, p.part_ml[((base + s) * p.R_pad + r) * 2]);
-    float l_all = 0.f, o = 0.f;
+    for (int s = 0; s < p.n_splits; ++s) m_all = fmaxf(m_all, ml[(base + s) * p.R_pad + r].x);
+    float l_all = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
     for (int s = 0; s < p.n_splits; ++s) {
         const size_t prow = (base + s) * p.R_pad + r;
-        const float m_s = p.part_ml[prow * 2];
-        if (m_s == -INFINITY) continue;
-        const float w = __expf(m_s - m_all);
-        l_all = fmaf(p.part_ml[prow * 2 + 1], w, l_all);
-        o = fmaf(p.part_o[prow * kD + c], w, o);
+        const float2 m_l = ml[prow];
+        if (m_l.x == -INFINITY) continue;  // an empty split: its partial O was never written
+        const float4 po = reinterpret_cast<const float4*>(p.part_o + prow * kD)[lane];
+        const float w = __expf(m_l.x - m_all);
+        l_all = fmaf(m_l.y, w, l_all);
+        o.x = fmaf(po.x, w, o.x);
+        o.y = fmaf(po.y, w, o.y);
+        o.z = fmaf(po.z, w, o.z);
+        o.w = fmaf(po.w, w, o.w);
     }
     const int j = r / p.G, g = r % p.G;
     const size_t row = ((size_t)lb * p.M_max + j) * p.Hq + h * p.G + g;
-    const float val = o / l_all;
-    if (p.out_f32) reinterpret_cast<float*>(p.out)[row * kD + c] = val;
-    else reinterpret_cast<__nv_bfloat16*>(p.out)[row * kD + c] = __float2bfloat16_rn(val);
-    if (p.lse && c == 0) p.lse[row] = m_all + logf(l_all);
+    const float inv = 1.f / l_all;
+    o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+    if (p.out_f32) {
+        reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + row * kD)[lane] = o;
+    } else {
+        uint2 w2;
+        w2.x = pack_bf16(o.x, o.y);
+        w2.y = pack_bf16(o.z, o.w);
+        reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + row * kD)[lane] = w2;
+    }
+    if (p.lse && lane == 0) p.lse[row] = m_all + logf(l_all);
 }
 
 }  // namespace
@@ -647,8 +663,8 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
     if (p.n_splits > 1) {
-        dim3 mgrid(R_max, Hkv, a.n_layers * a.batch);
-        merge_tc_kernel<<<mgrid, kD, 0, stream>>>(p);
+        dim3 mgrid((R_max + kMergeRows - 1) / kMergeRows, Hkv, a.n_layers * a.batch);
+        merge_tc_kernel<<<mgrid, 32 * kMergeRows, 0, stream>>>(p);
         if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
         count_launch();
     }

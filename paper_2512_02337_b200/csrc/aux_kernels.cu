@@ -11,11 +11,17 @@ namespace specpv {
 namespace {
 
 // ---------------------------------------------------------------------------------------------
-// Eq. 1: Kmax/Kmin per block.  grid = (blocks touched, Hkv, layers x seqs), one thread per channel.
+// Eq. 1: Kmax/Kmin per block.  grid = (blocks touched, Hkv, layers x seqs).  A thread owns one 16-byte
+// chunk of channels (kChunk of them) and every kTokLanes-th token of the block, with all its loads in
+// flight at once; the token lanes are then combined through shared memory.  max/min are exact, so the
+// order of the reduction does not matter.
 // ---------------------------------------------------------------------------------------------
+constexpr int kSumThreads = 128;
 template <typename T>
-__global__ void summaries_kernel(SummaryParams p) {
-    const int h = blockIdx.y, lb = blockIdx.z, c = threadIdx.x;
+__global__ void __launch_bounds__(kSumThreads) summaries_kernel(SummaryParams p) {
+    constexpr int kChunk = 16 / (int)sizeof(T);  // channels per 16-byte load
+    __shared__ float s_max[kSumThreads * kChunk], s_min[kSumThreads * kChunk];
+    const int h = blockIdx.y, lb = blockIdx.z, tid = threadIdx.x;
     const int b = lb % p.batch, l = lb / p.batch;
     int seq_len = p.seq_lens[b];
     if (p.n_appended) {  // summaries of a commit in flight: the lengths are not advanced yet
@@ -28,20 +34,57 @@ __global__ void summaries_kernel(SummaryParams p) {
     const int n_valid = min(p.bs, seq_len - i * p.bs);
     const int page = p.block_table[(size_t)b * p.max_blocks + i];
     if (page < 0 || page >= p.n_pages) {
-        if (c == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, i, page, l);
+        if (tid == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, i, page, l);
         return;
     }
     const T* k = reinterpret_cast<const T*>(p.k_pool) +
                  (((size_t)(p.layer0 + l) * p.n_pages + page) * p.Hkv + h) * p.bs * p.d;
-    float mx = -INFINITY, mn = INFINITY;
-    for (int t = 0; t < n_valid; ++t) {
-        float v = to_float(k[(size_t)t * p.d + c]);
-        mx = fmaxf(mx, v);
-        mn = fminf(mn, v);
+    const int chunks = p.d / kChunk;            // 16-byte chunks per token row (8, 16 or 32)
+    const int tok_lanes = kSumThreads / chunks;  // tokens read side by side
+    const int chunk = tid % chunks, tl = tid / chunks;
+    float mx[kChunk], mn[kChunk];
+#pragma unroll
+    for (int e = 0; e < kChunk; ++e) { mx[e] = -INFINITY; mn[e] = INFINITY; }
+    constexpr int kMaxIter = 16;  // bs <= 64 and tok_lanes >= 4
+    uint4 buf[kMaxIter];
+    int n_it = 0;
+#pragma unroll
+    for (int it = 0; it < kMaxIter; ++it) {
+        const int t = tl + it * tok_lanes;
+        if (t < n_valid) {
+            buf[it] = *reinterpret_cast<const uint4*>(k + (size_t)t * p.d + chunk * kChunk);
+            n_it = it + 1;
+        }
     }
-    const size_t o = ((((size_t)(p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks + i) * p.d + c;
-    reinterpret_cast<T*>(p.kmax)[o] = from_float<T>(mx);
-    reinterpret_cast<T*>(p.kmin)[o] = from_float<T>(mn);
+#pragma unroll
+    for (int it = 0; it < kMaxIter; ++it) {
+        if (it < n_it) {
+            const T* e8 = reinterpret_cast<const T*>(&buf[it]);
+#pragma unroll
+            for (int e = 0; e < kChunk; ++e) {
+                const float v = to_float(e8[e]);
+                mx[e] = fmaxf(mx[e], v);
+                mn[e] = fminf(mn[e], v);
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < kChunk; ++e) {
+        s_max[(tl * chunks + chunk) * kChunk + e] = mx[e];
+        s_min[(tl * chunks + chunk) * kChunk + e] = mn[e];
+    }
+    __syncthreads();
+    // thread c < d finishes channel c over the token lanes
+    for (int c = tid; c < p.d; c += kSumThreads) {
+        float a = -INFINITY, z = INFINITY;
+        for (int q = 0; q < tok_lanes; ++q) {
+            a = fmaxf(a, s_max[q * p.d + c]);
+            z = fminf(z, s_min[q * p.d + c]);
+        }
+        const size_t o = ((((size_t)(p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks + i) * p.d + c;
+        reinterpret_cast<T*>(p.kmax)[o] = from_float<T>(a);
+        reinterpret_cast<T*>(p.kmin)[o] = from_float<T>(z);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -327,8 +370,8 @@ specpv_status launch_summaries(const SummaryParams& p, int n_layers, int blocks_
                                cudaStream_t stream) {
     if (blocks_touched <= 0 || n_layers <= 0) return SPECPV_OK;
     dim3 grid(blocks_touched, p.Hkv, n_layers * p.batch);
-    if (dtype == SPECPV_DTYPE_F32) summaries_kernel<float><<<grid, p.d, 0, stream>>>(p);
-    else summaries_kernel<__nv_bfloat16><<<grid, p.d, 0, stream>>>(p);
+    if (dtype == SPECPV_DTYPE_F32) summaries_kernel<float><<<grid, kSumThreads, 0, stream>>>(p);
+    else summaries_kernel<__nv_bfloat16><<<grid, kSumThreads, 0, stream>>>(p);
     SPECPV_CHECK_LAUNCH();
     return SPECPV_OK;
 }

@@ -18,6 +18,12 @@ namespace {
 
 using namespace tc;
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 constexpr int kScoreThreads = 192;       // warp 0: TMA + MMA issue, warp 1: idle, warps 2-5: epilogue (lane quarters 2,3,0,1)
 constexpr int kTileBlocks = 128;
 constexpr int kSumTileBytes = 32768;     // [2 d-halves][128 blocks][64 d] bf16
@@ -82,7 +88,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
             mbar_init(smem_u32(&bars.sum_empty[s]), 1);
         }
         mbar_init(smem_u32(&bars.d_full), 1);
-        mbar_init(smem_u32(&bars.d_empty), 128);
+        mbar_init(smem_u32(&bars.d_empty), 4);  // one arrival per epilogue warp
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -100,57 +106,66 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     const uint32_t idesc = make_idesc((uint32_t)p.n_cols, false);
 
     if (warp == 0) {
+        // ---- producer + MMA issue: the whole warp runs the loop (a lone lane of a diverged warp runs
+        // slowly), lane 0 issues ----------------------------------------------------------------------
+        const uint32_t qbar = smem_u32(&bars.q_full);
+        const int n_q_tiles = p.n_cols > 128 ? 2 : 1;
+        const int row0 = (((p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks;
+        auto load_tile = [&](int i) {  // lane 0 only
+            const int slot = i % kScoreStages;
+            const uint32_t full = smem_u32(&bars.sum_full[slot]);
+            mbar_expect_tx(full, 2 * kSumTileBytes);
+            const uint32_t dst = sum_smem + slot * 2 * kSumTileBytes;
+            const int row = row0 + (tile_begin + i) * kTileBlocks;
+            for (int half = 0; half < 2; ++half) {
+                tma_load_2d(dst + half * 16384, &p.tm_kmax, half * 64, row, full);
+                tma_load_2d(dst + kSumTileBytes + half * 16384, &p.tm_kmin, half * 64, row, full);
+            }
+        };
         if (lane == 0) {
-            // ---- producer + MMA issue (one thread) -------------------------------------------------
-            const uint32_t qbar = smem_u32(&bars.q_full);
-            const int n_q_tiles = p.n_cols > 128 ? 2 : 1;
             mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
             for (int t = 0; t < n_q_tiles; ++t)
                 for (int half = 0; half < 2; ++half)
                     tma_load_3d(q_smem + half * 32768 + t * 16384, &p.tm_q, half * 64, h * p.G,
                                 lb * p.M_max + t * tok_per_tile, qbar);
-            const int row0 = (((p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks;
-            auto load_tile = [&](int i) {
-                const int slot = i % kScoreStages;
-                const uint32_t full = smem_u32(&bars.sum_full[slot]);
-                mbar_expect_tx(full, 2 * kSumTileBytes);
-                const uint32_t dst = sum_smem + slot * 2 * kSumTileBytes;
-                const int row = row0 + (tile_begin + i) * kTileBlocks;
-                for (int half = 0; half < 2; ++half) {
-                    tma_load_2d(dst + half * 16384, &p.tm_kmax, half * 64, row, full);
-                    tma_load_2d(dst + kSumTileBytes + half * 16384, &p.tm_kmin, half * 64, row, full);
-                }
-            };
             load_tile(0);
-            bool ok = mbar_wait(qbar, 0, abort_flag, p.workspace, 20);
-            for (int i = 0; ok && i < n_tiles; ++i) {
-                if (i + 1 < n_tiles) {
-                    const int use = i + 1;
-                    if (use >= kScoreStages)
-                        ok = mbar_wait(smem_u32(&bars.sum_empty[use % kScoreStages]), ((use / kScoreStages) - 1) & 1,
-                                       abort_flag, p.workspace, 21);
-                    if (!ok) break;
-                    load_tile(use);
-                }
-                const int slot = i % kScoreStages;
-                ok = mbar_wait(smem_u32(&bars.sum_full[slot]), (i / kScoreStages) & 1, abort_flag, p.workspace, 22);
-                if (!ok) break;
-                if (i > 0) ok = mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_max = sum_smem + slot * 2 * kSumTileBytes, a_min = a_max + kSumTileBytes;
+        }
+        __syncwarp();
+        // descriptors: constant upper word (8-row group stride 1024 B, version, 128-byte swizzle); lower word =
+        // 16-byte address, leading offset 16 B
+        const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
+        const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | (1u << 16);
+        const uint32_t sum_lo = ((sum_smem >> 4) & 0x3FFFu) | (1u << 16);
+        bool ok = mbar_wait(qbar, 0, abort_flag, p.workspace, 20);
+        for (int i = 0; i < n_tiles; ++i) {
+            if (i + 1 < n_tiles) {
+                const int use = i + 1;
+                if (use >= kScoreStages)
+                    ok &= mbar_wait(smem_u32(&bars.sum_empty[use % kScoreStages]), ((use / kScoreStages) - 1) & 1,
+                                    abort_flag, p.workspace, 21);
+                if (lane == 0 && ok) load_tile(use);
+                __syncwarp();
+            }
+            const int slot = i % kScoreStages;
+            ok &= mbar_wait(smem_u32(&bars.sum_full[slot]), (i / kScoreStages) & 1, abort_flag, p.workspace, 22);
+            if (i > 0) ok &= mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t a_max = sum_lo + (uint32_t)slot * (2 * kSumTileBytes >> 4), a_min = a_max + (kSumTileBytes >> 4);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t a_off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                    const uint32_t b_off = (kk >> 2) * 32768 + (kk & 3) * 32;
-                    const uint64_t bdesc = make_desc(q_smem + b_off, 16, 1024);
-                    mma_ss(tmem, make_desc(a_max + a_off, 16, 1024), bdesc, idesc, kk > 0);
-                    mma_ss(tmem + 256, make_desc(a_min + a_off, 16, 1024), bdesc, idesc, kk > 0);
+                    const uint32_t a_off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                    const uint32_t b_off = (uint32_t)((kk >> 2) * 32768 + (kk & 3) * 32) >> 4;
+                    const uint64_t bdesc = ((uint64_t)desc_hi << 32) | (q_lo + b_off);
+                    mma_ss(tmem, ((uint64_t)desc_hi << 32) | (a_max + a_off), bdesc, idesc, kk > 0);
+                    mma_ss(tmem + 256, ((uint64_t)desc_hi << 32) | (a_min + a_off), bdesc, idesc, kk > 0);
                 }
                 tc_commit(smem_u32(&bars.d_full));
                 tc_commit(smem_u32(&bars.sum_empty[slot]));
             }
+            __syncwarp();
         }
+        (void)ok;
     } else if (warp >= 2) {
         // ---- epilogue: thread <-> block of the tile -----------------------------------------------
         const int q = warp & 3;  // tensor-memory lane quarter of this warp
@@ -161,21 +176,41 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
             ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full), i & 1, abort_flag, p.workspace, 24));
             if (!ok) break;
             tc_fence_after();
-            float red = p.reduce == SPECPV_REDUCE_MAX ? -INFINITY : 0.f;
-            for (int c0 = (col_begin / 32) * 32; c0 < col_end; c0 += 32) {
-                uint32_t vmax[32], vmin[32];
-                TMEM_LD32(tmem + lane_addr + c0, vmax);
-                TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
-                tmem_wait_ld();
+            // four independent partial reductions: a single chain through one register would leave this
+            // warp, alone on its scheduler, waiting out the latency of every instruction
+            const bool is_max = p.reduce == SPECPV_REDUCE_MAX;
+            float r4[4];
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    const int c = c0 + k;
-                    const float s = fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
-                    if (c >= col_begin && c < col_end) red = p.reduce == SPECPV_REDUCE_MAX ? fmaxf(red, s) : red + s;
+            for (int e = 0; e < 4; ++e) r4[e] = is_max ? -INFINITY : 0.f;
+            for (int c0 = (col_begin / 64) * 64; c0 < col_end; c0 += 64) {
+                uint32_t vmax[64], vmin[64];
+                TMEM_LD32(tmem + lane_addr + c0, vmax);
+                TMEM_LD32(tmem + lane_addr + c0 + 32, (vmax + 32));
+                TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
+                TMEM_LD32(tmem + lane_addr + 256 + c0 + 32, (vmin + 32));
+                tmem_wait_ld();
+                const bool whole = c0 >= col_begin && c0 + 64 <= col_end;  // warp-uniform
+                if (whole && !is_max) {
+#pragma unroll
+                    for (int k = 0; k < 64; ++k)
+                        r4[k & 3] += fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
+                } else if (whole) {
+#pragma unroll
+                    for (int k = 0; k < 64; ++k)
+                        r4[k & 3] = fmax3(r4[k & 3], __uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 64; ++k) {
+                        const int c = c0 + k;
+                        const float sc = fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
+                        if (c >= col_begin && c < col_end) r4[k & 3] = is_max ? fmaxf(r4[k & 3], sc) : r4[k & 3] + sc;
+                    }
                 }
             }
+            float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars.d_empty));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty));
             const int blk = (tile_begin + i) * kTileBlocks + blk_in_tile;
             if (blk < nb) {
                 if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)(col_end - col_begin);
