@@ -37,6 +37,16 @@ METRIC = "verify_attention_us_per_step"
 ACCEPT_LEN = 4  # tokens committed per step: the paper's mean accept length is 3.3-3.6 (Table 1), plus the root
 
 
+# DRAM bytes (read + write) of one full-verification attention launch per layer, from the ncu capture of the
+# 2-layer case summarised in profiles/attn_tc_kernel_llama_128k.md; the traffic is proportional to the layers streamed.
+NCU_DRAM_BYTES_PER_LAYER = {"llama_128k": (1.075371e9 + 6.274816e6) / 2}
+
+
+def ncu_traffic_bytes(workload: str, n_layers: int):
+    per_layer = NCU_DRAM_BYTES_PER_LAYER.get(workload)
+    return None if per_layer is None else per_layer * n_layers
+
+
 def load_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -340,7 +350,7 @@ def main():
                 "peak": peaks["hbm_gbs"] if bound == "hbm" else peaks["bf16_tflops"],
                 "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
                 "frac": (achieved_gbs / peaks["hbm_gbs"]) if bound == "hbm" else achieved_tf / peaks["bf16_tflops"],
-                "peak_source": peaks["source"], "traffic": None,
+                "peak_source": peaks["source"], "traffic": ncu_traffic_bytes(args.workload, st["L"]),
                 "launch_us": full_avg_s * 1e6, "bound_us": max(t_hbm, t_tensor) * 1e6,
                 "achieved_gbs": achieved_gbs, "achieved_tflops": achieved_tf,
                 "frac_of_bound": max(t_hbm, t_tensor) / full_avg_s}
