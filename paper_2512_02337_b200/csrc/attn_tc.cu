@@ -387,16 +387,19 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 // scaling the output).
                 auto exp_row = [&](float m_use) {
                     const float2 nm2 = make_float2(-m_use, -m_use);
-                    float2 sum2 = make_float2(0.f, 0.f);
+                    float2 sum2[4];  // independent partial sums: one chain of 64 dependent adds would outlast the exponentials
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) sum2[e] = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int i = 0; i < 64; ++i) {
                         const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])),
                                                     sc2, nm2);
                         const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
                         v[i] = w;
-                        sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+                        sum2[i & 3] = __fadd2_rn(sum2[i & 3], make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
                     }
-                    return sum2.x + sum2.y;
+                    const float2 s01 = __fadd2_rn(sum2[0], sum2[1]), s23 = __fadd2_rn(sum2[2], sum2[3]);
+                    return (s01.x + s23.x) + (s01.y + s23.y);
                 };
                 // Fast path (every full context tile after the first): keep the reference m_run of the row as it
                 // is and skip the row maximum.  Weights may then exceed 1; float32 sums and bf16 weights keep
