@@ -48,6 +48,7 @@ def _load():
         _lib.oracle_num_threads.restype = ctypes.c_int
         _lib.oracle_block_summaries.restype = None
         _lib.oracle_block_scores.restype = None
+        _lib.oracle_block_scores_mode.restype = None
         _lib.oracle_tree_attention.restype = None
     return _lib
 
@@ -106,16 +107,18 @@ def block_summaries(k_pool, block_table, seq_len: int):
     return kmax, kmin
 
 
-def block_scores(q, kmax, kmin, Hkv: int, reduce: int = 0, last_query: int = 0) -> np.ndarray:
-    """Eq. 2-3.  q [M][Hq][d]; kmax/kmin [Hkv][nb][d] f64 -> scores [Hkv][nb] f64."""
+def block_scores(q, kmax, kmin, Hkv: int, reduce: int = 0, last_query: int = 0, score_mode: int = 0) -> np.ndarray:
+    """Eq. 2-3.  q [M][Hq][d]; kmax/kmin [Hkv][nb][d] f64 -> scores [Hkv][nb] f64.
+
+    score_mode 0 is Eq. 2 as printed; 1 is the channel-wise form sum_c max(q_c Kmax_c, q_c Kmin_c)."""
     q = _c(q)
     M, Hq, d = q.shape
     kmax = _c(kmax, np.float64)
     kmin = _c(kmin, np.float64)
     nb = kmax.shape[1]
     scores = np.empty((Hkv, nb), dtype=np.float64)
-    _load().oracle_block_scores(_p(q), _code(q), M, Hq, Hkv, d, _p(kmax), _p(kmin), nb,
-                                reduce, last_query, _p(scores))
+    _load().oracle_block_scores_mode(_p(q), _code(q), M, Hq, Hkv, d, _p(kmax), _p(kmin), nb,
+                                     reduce, last_query, score_mode, _p(scores))
     return scores
 
 

@@ -127,9 +127,9 @@ ORACLE_API void oracle_block_summaries(const void *k_pool, int dtype, int Hkv, i
  * Eq. 2-3: s_{i,j} = max(q_j . Kmax_i, q_j . Kmin_i), reduced over the step's query rows.
  * reduce: 0 mean, 1 max, 2 last (row `last_query`, averaged over the G heads of the group).
  * ------------------------------------------------------------------------------------------ */
-ORACLE_API void oracle_block_scores(const void *q, int dtype, int M, int Hq, int Hkv, int d,
-                                    const double *kmax, const double *kmin, int nb,
-                                    int reduce, int last_query, double *scores) {
+ORACLE_API void oracle_block_scores_mode(const void *q, int dtype, int M, int Hq, int Hkv, int d,
+                                         const double *kmax, const double *kmin, int nb,
+                                         int reduce, int last_query, int score_mode, double *scores) {
     int G = Hq / Hkv;
 #pragma omp parallel for collapse(2) schedule(static)
     for (int h = 0; h < Hkv; ++h)
@@ -142,13 +142,18 @@ ORACLE_API void oracle_block_scores(const void *q, int dtype, int M, int Hq, int
                 if (reduce == 2 && j != last_query) continue;
                 for (int g = 0; g < G; ++g) {
                     int64_t qoff = ((int64_t)j * Hq + h * G + g) * d;
-                    double dmax = 0.0, dmin = 0.0;
+                    double dmax = 0.0, dmin = 0.0, chan = 0.0;
                     for (int c = 0; c < d; ++c) {
                         double qc = load_elem(q, dtype, qoff + c);
-                        dmax += qc * bmax[c];
-                        dmin += qc * bmin[c];
+                        double a = qc * bmax[c], b = qc * bmin[c];
+                        dmax += a;
+                        dmin += b;
+                        chan += a > b ? a : b;  /* channel-wise form: the maximum is taken per channel */
                     }
-                    double s = dmax > dmin ? dmax : dmin;
+                    /* score_mode 0: Eq. 2 as printed (max of the two full dot products);
+                     * score_mode 1: the channel-wise bound of Quest, which Section 3.2 cites as its inspiration:
+                     *               sum_c max(q_c Kmax_c, q_c Kmin_c) >= q . k for every key k of the block */
+                    double s = score_mode == 1 ? chan : (dmax > dmin ? dmax : dmin);
                     if (reduce == 1) { if (s > acc) acc = s; }
                     else acc += s;
                     ++count;
@@ -156,6 +161,12 @@ ORACLE_API void oracle_block_scores(const void *q, int dtype, int M, int Hq, int
             }
             scores[(size_t)h * nb + i] = reduce == 1 ? acc : acc / (double)count;
         }
+}
+
+ORACLE_API void oracle_block_scores(const void *q, int dtype, int M, int Hq, int Hkv, int d,
+                                    const double *kmax, const double *kmin, int nb,
+                                    int reduce, int last_query, double *scores) {
+    oracle_block_scores_mode(q, dtype, M, Hq, Hkv, d, kmax, kmin, nb, reduce, last_query, 0, scores);
 }
 
 /* ------------------------------------------------------------------------------------------

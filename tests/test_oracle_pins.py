@@ -131,6 +131,35 @@ def test_block_scores_match_independent_einsum(reduce):
     np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
 
 
+def test_channelwise_scores_closed_form_bound_and_separation():
+    """score_mode 1 (the channel-wise form of Quest, cited by Section 3.2): three pins that do not retype it."""
+    rng = np.random.default_rng(21)
+    M, Hq, Hkv, d, nb, bs = 5, 4, 2, 16, 6, 8
+    G = Hq // Hkv
+    q = rng.standard_normal((M, Hq, d)).astype(np.float32)
+    keys = rng.standard_normal((Hkv, nb, bs, d))
+    kmax, kmin = keys.max(axis=2), keys.min(axis=2)
+    got = oracle.block_scores(q, kmax, kmin, Hkv, reduce=1, score_mode=1)  # max over the rows
+    qw = q.astype(np.float64).reshape(M, Hkv, G, d)
+    # (a) sign split: for q_c >= 0 the channel takes Kmax, for q_c < 0 it takes Kmin, so the score is two plain
+    #     contractions, q+ . Kmax + q- . Kmin
+    split = np.einsum("mhgc,hic->hmgi", np.maximum(qw, 0), kmax) + np.einsum("mhgc,hic->hmgi", np.minimum(qw, 0), kmin)
+    np.testing.assert_allclose(got, split.max(axis=(1, 2)), rtol=1e-12, atol=1e-12)
+    # (b) it bounds the true score of every key of the block from above (the reason Quest uses it)
+    true = np.einsum("mhgc,hitc->hmgit", qw, keys)
+    assert np.all(split[..., None] >= true - 1e-12)
+    # (c) it is never below Eq. 2 as printed, and strictly above when the channels disagree in sign
+    printed = oracle.block_scores(q, kmax, kmin, Hkv, reduce=1, score_mode=0)
+    assert np.all(got >= printed - 1e-12) and np.any(got > printed + 1e-6)
+    one = oracle.block_scores(np.array([[[1.0, -1.0]]], dtype=np.float32), np.array([[[1.0, 1.0]]]),
+                              np.array([[[0.0, 0.0]]]), 1, score_mode=1)
+    assert one[0, 0] == 1.0  # 1*1 + max(-1*1, -1*0) = 1, where the printed form gives 0
+    # blocks of one repeated key: both forms equal q . k
+    same = np.repeat(keys[:, :, :1], bs, axis=2)
+    eq = oracle.block_scores(q, same.max(axis=2), same.min(axis=2), Hkv, reduce=0, score_mode=1)
+    np.testing.assert_allclose(eq, np.einsum("mhgc,hic->hmgi", qw, same[:, :, 0]).mean(axis=(1, 2)), rtol=1e-12, atol=1e-12)
+
+
 def test_block_scores_is_max_of_full_dot_products_not_channelwise():
     # q = (1, -1), Kmax = (1, 1), Kmin = (0, 0): Eq. 2 as printed gives max(0, 0) = 0,
     # the channel-wise variant would give 1*1 + (-1)*0 = 1.
