@@ -79,7 +79,8 @@ typedef struct {
     int32_t budget_blocks; /* sink + retrieval + local blocks of the partial cache */
     int32_t buffer_tokens; /* extra room after the budget for partially verified + candidate tokens */
     int32_t reduce;        /* SPECPV_REDUCE_*: the f of Eq. 3 */
-    int32_t score_mode;    /* 0 = Eq. 2 as printed (max of the two full dot products) */
+    int32_t score_mode;    /* 0 = Eq. 2 as printed (max of the two full dot products); 1 = the channel-wise
+                              form sum_c max(q_c Kmax_c, q_c Kmin_c) of the method Section 3.2 cites */
     float softmax_scale;   /* 0 => 1/sqrt(head_dim) */
     int32_t out_f32;       /* 1 => the attention output O is written as float32 whatever dtype is
                               (the accumulator before the final rounding); 0 => O has type dtype */
@@ -137,7 +138,9 @@ specpv_status specpv_update_block_summaries(const specpv_config *cfg, int layer0
 
 /* Eq. 2-3: scores[l][b][h][i] = f_j max(q_j . Kmax_i, q_j . Kmin_i) over the step's query rows of
  * KV head h's group (all G heads x q_lens[b] tokens; for SPECPV_REDUCE_LAST the G heads of row
- * last_query[b] (device [batch], NULL = row 0)).  Blocks >= ceil(seq_len/bs) are left untouched. */
+ * last_query[b] (device [batch], NULL = row 0)).  With cfg->score_mode = 1 the maximum is taken per channel
+ * before the sum (an upper bound of q . k over the block's keys).  Blocks >= ceil(seq_len/bs) are left
+ * untouched. */
 specpv_status specpv_score_blocks(const specpv_config *cfg, int layer0, int n_layers, const void *q,
                                   const int32_t *q_lens, int M_max, const int32_t *last_query,
                                   const void *kmax, const void *kmin, const specpv_paged_kv *kv,

@@ -27,7 +27,7 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     if (cfg->sink_blocks < 0 || cfg->local_blocks < 1 || cfg->buffer_tokens < 0) return SPECPV_ERR_BUDGET;
     if (cfg->budget_blocks < cfg->sink_blocks + cfg->local_blocks + 1) return SPECPV_ERR_BUDGET;
     if (cfg->reduce < 0 || cfg->reduce > 2) return SPECPV_ERR_INVALID_ARG;
-    if (cfg->score_mode != 0) return SPECPV_ERR_UNSUPPORTED;
+    if (cfg->score_mode != 0 && cfg->score_mode != 1) return SPECPV_ERR_UNSUPPORTED;
     if (cfg->out_f32 != 0 && cfg->out_f32 != 1) return SPECPV_ERR_INVALID_ARG;
     if (!(cfg->softmax_scale >= 0.f) || isinf(cfg->softmax_scale)) return SPECPV_ERR_INVALID_ARG;
     g->n_layers = cfg->n_layers;
@@ -45,6 +45,7 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     g->budget_blocks = cfg->budget_blocks;
     g->buffer_tokens = cfg->buffer_tokens;
     g->reduce = cfg->reduce;
+    g->score_mode = cfg->score_mode;
     g->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
     return SPECPV_OK;
 }
@@ -236,8 +237,10 @@ SPECPV_EXPORT specpv_status specpv_score_blocks(const specpv_config* cfg, int la
     p.scores = scores; p.layer0 = layer0; p.batch = kv->batch; p.M_max = M_max; p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
     p.bs = g.bs; p.max_blocks = kv->max_blocks; p.reduce = g.reduce;
     p.workspace = workspace;
+    p.score_mode = g.score_mode;
     const int max_nb = (kv->max_seq_len + g.bs - 1) / g.bs;
-    if (scores_tc_supported(g.dtype, g.d, g.G, M_max) && aligned16(q) && aligned16(kmax) && aligned16(kmin))
+    // the tensor-core kernel computes Eq. 2 as printed; the channel-wise form runs on the SIMT kernel
+    if (g.score_mode == 0 && scores_tc_supported(g.dtype, g.d, g.G, M_max) && aligned16(q) && aligned16(kmax) && aligned16(kmin))
         return launch_scores_tc(p, n_layers, g.n_layers, max_nb, reinterpret_cast<cudaStream_t>(stream));
     return launch_scores(p, n_layers, max_nb, g.dtype, g.d, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -150,15 +150,31 @@ __global__ void __launch_bounds__(32 * kScoreWarps) scores_simt_kernel(ScorePara
         float dmax[kScoreRowTile], dmin[kScoreRowTile];
 #pragma unroll
         for (int i = 0; i < kScoreRowTile; ++i) dmax[i] = dmin[i] = 0.f;
+        if (p.score_mode == 0) {
 #pragma unroll 4
-        for (int c = 0; c < D; ++c) {
-            float a = my_max[c], bb = my_min[c];
+            for (int c = 0; c < D; ++c) {
+                float a = my_max[c], bb = my_min[c];
 #pragma unroll
-            for (int i = 0; i < kScoreRowTile; ++i) {
-                float qc = Qs[i * D + c];
-                dmax[i] = fmaf(qc, a, dmax[i]);
-                dmin[i] = fmaf(qc, bb, dmin[i]);
+                for (int i = 0; i < kScoreRowTile; ++i) {
+                    float qc = Qs[i * D + c];
+                    dmax[i] = fmaf(qc, a, dmax[i]);
+                    dmin[i] = fmaf(qc, bb, dmin[i]);
+                }
             }
+        } else {
+            // channel-wise form: a channel with q_c >= 0 takes Kmax_c, one with q_c < 0 takes Kmin_c
+            // (Kmax_c >= Kmin_c), so the score is one dot product with a per-channel choice of operand
+#pragma unroll 4
+            for (int c = 0; c < D; ++c) {
+                float a = my_max[c], bb = my_min[c];
+#pragma unroll
+                for (int i = 0; i < kScoreRowTile; ++i) {
+                    float qc = Qs[i * D + c];
+                    dmax[i] = fmaf(qc, qc < 0.f ? bb : a, dmax[i]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kScoreRowTile; ++i) dmin[i] = dmax[i];
         }
 #pragma unroll
         for (int i = 0; i < kScoreRowTile; ++i) {

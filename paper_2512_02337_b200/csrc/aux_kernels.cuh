@@ -26,6 +26,7 @@ struct ScoreParams {
     float* scores;
     void* workspace;
     int layer0, batch, M_max, Hq, Hkv, G, bs, max_blocks, reduce;
+    int score_mode;  // 0: max of the two full dot products (Eq. 2 as printed), 1: maximum per channel
 };
 
 struct SelectParams {

@@ -135,18 +135,28 @@ def test_qwen3_64k_decode_loop_64_steps():
     """Config "qwen3_64k_loop": 36 layers, 64K context, 48-node trees, 64 steps; partial verification
     every step, full verification with refresh every 8th step over the chain of partially verified tokens
     plus the tree, accepted path lengths 1..6 drawn from the seed.  An oracle loop mirrors layers 0 and 35."""
+    run_decode_loop("qwen3_64k_loop", n_steps=64, period=8)
+
+
+def test_decode_loop_paper_geometry_refresh_on_buffer_overflow():
+    """The paper's own settings (Appendix "Generation Settings"): 16-token blocks, 32 sink and 128 local tokens,
+    a 512-token budget and a buffer of 20 tokens beyond the tree; the refresh is triggered by the mode rule
+    alone (partially verified + candidate tokens exceed the buffer), not by a fixed period."""
+    run_decode_loop("llama_32k", n_steps=24, period=None, n_layers=2, ctx=[16 * 300 + 7], bs=16, M=12, depth=4,
+                    branch=3, budget_blocks=32, buffer_tokens=20 + 12)
+
+
+def run_decode_loop(name, n_steps, period, **over):
     dev = torch.device("cuda")
-    name = "qwen3_64k_loop"
     c0 = wl.CONFIGS[name]
-    n_steps, period = 64, 8
     spare = n_steps * 6 + 64
-    w = wl.make_workload(name, device=dev, spare_tokens=spare)
+    w = wl.make_workload(name, device=dev, spare_tokens=spare, **over)
     c = w.cfg
     L, Hq, Hkv, d, bs, M = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"]
     rng = np.random.default_rng(c0["index"])
     cfg = util.config_for(w)
     sink, local, budget = cfg.sink_blocks, cfg.local_blocks, cfg.budget_blocks
-    M_max = (period - 1) * 6 + M  # the longest chain of partially verified tokens plus the tree
+    M_max = min(cfg.buffer_tokens + 6, 128)  # the longest chain of partially verified tokens plus the tree
     full = util.full_cache(w)
     full.max_seq_len = int(c["ctx"][0]) + spare
     ws = B.new_workspace(cfg, L, 1, full.max_seq_len, M_max)
@@ -166,7 +176,7 @@ def test_qwen3_64k_decode_loop_64_steps():
     B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax, kmin, ws)
 
     # the oracle's mirror of two layers
-    mirror = [0, L - 1]
+    mirror = sorted({0, L - 1})
     table = w.block_table[0].cpu().numpy()
     ptab = ptable[0].cpu().numpy()
     o_k = {l: wl.to_numpy(w.k_pool[l]).copy() for l in mirror}
@@ -181,15 +191,16 @@ def test_qwen3_64k_decode_loop_64_steps():
     pending = []  # per partially verified token: nothing but a count is needed on the GPU side
     for step in range(1, n_steps + 1):
         parents = wl.make_tree(M, c["depth"], c["branch"], rng)
-        accept_len = int(rng.integers(1, 7))
+        accept_len = int(rng.integers(1, min(6, c["depth"] + 1) + 1))
         depth = [len(wl.path_to(parents, n)) for n in range(M)]
         path = wl.path_to(parents, depth.index(accept_len))  # the accepted root-to-node path
         n_pv = len(pending)
         mode = B.specpv_select_mode(o_len, budget * bs, n_pv, M, cfg.buffer_tokens, initialised)
-        refresh = (step % period == 0) or not initialised
         assert mode in (B.MODE_REFRESH, B.MODE_PARTIAL)
-        if mode == B.MODE_REFRESH:
-            assert refresh  # the buffer is sized so that the rule never forces an earlier refresh
+        assert mode == oracle.select_mode(o_len, budget * bs, n_pv, M, cfg.buffer_tokens, initialised)
+        refresh = mode == B.MODE_REFRESH or (period is not None and step % period == 0)
+        if period is not None and mode == B.MODE_REFRESH:
+            assert step % period == 0 or not initialised  # the buffer is sized so that the rule never forces an earlier refresh
         n_chain = n_pv if refresh else 0
         m_rows = n_chain + M
         q = torch.randn((L, 1, M_max, Hq, d), generator=g, device=dev).to(torch.bfloat16)
@@ -266,4 +277,4 @@ def test_qwen3_64k_decode_loop_64_steps():
             o_plen = o_new
             assert int(plens[0]) == o_plen
             pending.extend([0] * len(acc))
-    assert o_len > int(c["ctx"][0]) + n_steps  # the cache has grown by the accepted tokens
+    assert o_len > int(c["ctx"][0]) and initialised  # the cache has grown by the accepted tokens

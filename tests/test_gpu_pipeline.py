@@ -13,12 +13,12 @@ from tests import util
 pytestmark = pytest.mark.gpu
 
 
-def run_pipeline(name, n_layers=None, reduce=0, **over):
+def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, **over):
     w = wl.make_workload(name, device="cuda", n_layers=n_layers, spare_tokens=256, **over)
     c = w.cfg
     L, Hq, Hkv, d, bs, M = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"]
     batch = w.batch
-    cfg = util.config_for(w, reduce=reduce)
+    cfg = util.config_for(w, reduce=reduce, score_mode=score_mode)
     full = util.full_cache(w)
     full.max_seq_len = int(max(c["ctx"])) + 256
     ws = B.new_workspace(cfg, L, batch, full.max_seq_len, M)
@@ -53,7 +53,7 @@ def run_pipeline(name, n_layers=None, reduce=0, **over):
     B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, out_full, lse_full, ws)
     B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, out_part, lse_part, ws)
     if c["dtype"] == "bf16":  # the bfloat16 output is the float32 one, rounded
-        cfg16 = util.config_for(w, reduce=reduce, out_f32=0)
+        cfg16 = util.config_for(w, reduce=reduce, score_mode=score_mode, out_f32=0)
         o16f, o16p = torch.zeros_like(out_full, dtype=dt), torch.zeros_like(out_full, dtype=dt)
         B.specpv_verify_full(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, o16f, None, ws)
         B.specpv_verify_partial(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, o16p, None, ws)
@@ -75,7 +75,7 @@ def run_pipeline(name, n_layers=None, reduce=0, **over):
             nb = (sl + bs - 1) // bs
             okmax, okmin = oracle.block_summaries(kp[l], table[b], sl)
             assert np.array_equal(kmax_g[l, b, :, :nb], okmax) and np.array_equal(kmin_g[l, b, :, :nb], okmin)
-            osc = oracle.block_scores(qn[l, b], okmax, okmin, Hkv, reduce=reduce, last_query=0)
+            osc = oracle.block_scores(qn[l, b], okmax, okmin, Hkv, reduce=reduce, last_query=0, score_mode=score_mode)
             np.testing.assert_allclose(scores_g[l, b, :, :nb], osc, rtol=2e-3 if c["dtype"] == "bf16" else 2e-5,
                                        atol=2e-2 if c["dtype"] == "bf16" else 2e-4)
             assert np.all(np.isnan(scores_g[l, b, :, nb:]))  # untouched beyond the context
@@ -122,6 +122,13 @@ def test_small_bf16_llama_shape_pipeline():
 def test_small_bf16_other_reductions(reduce):
     # max / last reductions through the tensor-core score kernel, M = 20 (80 query rows: one Q tile)
     run_pipeline("llama_32k", n_layers=1, reduce=reduce, ctx=[64 * 150 + 11], M=20)
+
+
+@pytest.mark.parametrize("reduce", [0, 1])
+def test_channelwise_score_mode_fp32_and_bf16(reduce):
+    # score_mode 1: the maximum is taken per channel; selection, gather and partial verification follow from it
+    run_pipeline("tiny_fp32", reduce=reduce, score_mode=1)
+    run_pipeline("llama_32k", n_layers=1, reduce=reduce, score_mode=1, ctx=[64 * 90 + 3], M=33)
 
 
 def test_ragged_batch_shuffled_table_pipeline():

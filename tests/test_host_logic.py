@@ -68,7 +68,7 @@ def test_config_validation_happens_on_the_host():
                 local_blocks=2, budget_blocks=8, buffer_tokens=64)
     assert B.specpv_workspace_bytes(B.make_config(**good), 2, 1, 2048, 16) > 256
     for key, val in [("n_q_heads", 7), ("head_dim", 96), ("block_tokens", 48), ("dtype", 5), ("budget_blocks", 3),
-                     ("local_blocks", 0), ("reduce", 3), ("score_mode", 1), ("softmax_scale", -1.0)]:
+                     ("local_blocks", 0), ("reduce", 3), ("score_mode", 2), ("softmax_scale", -1.0)]:
         assert B.specpv_workspace_bytes(B.make_config(**{**good, key: val}), 2, 1, 2048, 16) == 0, key
     # null pointers / bad layer ranges are refused before any CUDA call (works without a GPU)
     cfg = B.make_config(**good)
