@@ -83,6 +83,14 @@ __device__ __forceinline__ uint32_t launder(uint32_t x) {
     asm volatile("" : "+r"(x));
     return x;
 }
+// acc.x += low bf16 of w, acc.y += high bf16 of w: the mixed-precision add takes the 16-bit halves as they
+// are, so the packed word needs no shift / mask to be widened first (the sums are the same bit for bit)
+__device__ __forceinline__ void add_bf16_pair(float2& acc, uint32_t w) {
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\t"
+        "add.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+        : "+f"(acc.x), "+f"(acc.y)
+        : "r"(w));
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -396,7 +404,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                                                     sc2, nm2);
                         const uint32_t w = pack_bf16(ex2(x.x), ex2(x.y));
                         v[i] = w;
-                        sum2[i & 3] = __fadd2_rn(sum2[i & 3], make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+                        add_bf16_pair(sum2[i & 3], w);
                     }
                     const float2 s01 = __fadd2_rn(sum2[0], sum2[1]), s23 = __fadd2_rn(sum2[2], sum2[3]);
                     return (s01.x + s23.x) + (s01.y + s23.y);
