@@ -233,6 +233,55 @@ def timed_loop(st, steps, warmup, e2e, dist_barrier):
     return total_ms / steps, full_ms, part_ms, st["B"].specpv_kernel_launches() - launches0, (wall0, wall1)
 
 
+def max_over_ranks(values, device):
+    """Every rank's device-timed figures reduced with MAX (replicas run side by side: the job is as slow as
+    its slowest rank).  Works on any initialised process group (nccl on GPUs, gloo in the CPU test)."""
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def partial_budget_sweep(st, peaks, budgets=(32, 64, 128), iters=10):
+    """Partial verification alone for the partial budgets of the paper's sweep (2048 / 4096 / 8192 tokens at
+    64-token blocks): selection and gather with that budget (untimed), then the attention call timed with CUDA
+    events.  `frac` is against the HBM time of the bytes that call has to read (partial K/V + step tensors)."""
+    B, w, L, M, batch = st["B"], st["w"], st["L"], st["M"], st["batch"]
+    c = w.cfg
+    bs, Hkv, Hq, d = c["bs"], c["Hkv"], c["Hq"], c["d"]
+    dev = w.device
+    sink, local = wl.sink_local_blocks(bs)
+    out = []
+    for budget in budgets:
+        cfg = B.make_config(L, Hq, Hkv, d, bs, c["dtype"], sink, local, budget, c["buffer_tokens"])
+        idx = torch.zeros((L, batch, Hkv, budget), dtype=torch.int32, device=dev)
+        ppb = budget + (cfg.buffer_tokens + bs - 1) // bs + 1
+        pk = torch.zeros((L, batch * ppb, Hkv, bs, d), dtype=torch.bfloat16, device=dev)
+        plens = torch.zeros(batch, dtype=torch.int32, device=dev)
+        ptable = torch.arange(batch * ppb, dtype=torch.int32, device=dev).reshape(batch, ppb).contiguous()
+        partial = B.Cache(pk, torch.zeros_like(pk), ptable, plens, budget * bs + cfg.buffer_tokens)
+        B.specpv_select_partial_kv(cfg, L, st["scores"], w.seq_lens, batch, w.max_blocks, idx, st["count"], st["ws"])
+        B.specpv_refresh_partial(cfg, st["full"], idx, st["count"], partial, plens, st["ws"])
+        call = lambda: B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, st["mask"], None, M, partial,  # noqa: E731
+                                               st["out"], st["lse"], st["ws"])
+        for _ in range(3):
+            call()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        torch.cuda.synchronize(dev)
+        for a, b in ev:
+            a.record()
+            call()
+            b.record()
+        torch.cuda.synchronize(dev)
+        us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+        tokens = int(plens.sum())
+        nbytes = L * tokens * Hkv * 2 * d * 2 + L * batch * M * (2 * Hq + 2 * Hkv) * d * 2
+        out.append({"budget_tokens": budget * bs, "us": us, "bound_us": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                    "frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6)})
+        del pk, partial
+    return out
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -290,6 +339,7 @@ def main():
     ap.add_argument("--budget-blocks", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -328,12 +378,12 @@ def main():
     if not args.no_e2e:
         e2e_ms, _, _, _, _ = timed_loop(st, args.steps, warmup, True, barrier)
     if use_dist:
-        import torch.distributed as dist
-        t = torch.tensor([ms_step, e2e_ms if not args.no_e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, e2e_max = float(t[0]), float(t[1])
+        ms_step, e2e_max = max_over_ranks([ms_step, e2e_ms if not args.no_e2e else 0.0], dev)
         if not args.no_e2e:
             e2e_ms = e2e_max
+    sweep = None
+    if not args.no_sweep and rank == 0 and args.budget_blocks is None and c["dtype"] == "bf16":
+        sweep = partial_budget_sweep(st, load_peaks())
     if rank != 0:
         return 0
 
@@ -376,6 +426,8 @@ def main():
         h2d = 2 * (L * batch * M * (c["Hq"] + 2 * c["Hkv"]) * c["d"] * es + st["mask_host"].numel() * 8)
         d2h = 2 * (L * batch * M * c["Hq"] * (c["d"] * es + 4))
         out["e2e"] = {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    if sweep is not None:
+        out["partial_budget_sweep"] = sweep
     if not args.no_cpu_baseline and world == 1:
         us, sample, cores = oracle_sample(st)
         out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}

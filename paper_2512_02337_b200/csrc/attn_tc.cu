@@ -199,41 +199,46 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     if (warp == 0) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== TMA producer ================================================
+        // The whole warp runs the loop (a lone lane of a diverged warp runs slowly); lane 0 issues the copies.
+        const uint32_t qbar = smem_u32(&bars.q_full);
         if (lane == 0) {
-            const uint32_t qbar = smem_u32(&bars.q_full);
             mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
             for (int t = 0; t < n_q_tiles; ++t)
                 for (int half = 0; half < 2; ++half)
                     tma_load_3d(q_smem + t * 32768 + half * 16384, &p.tm_q, half * 64, h * p.G,
                                 lb * p.M_max + tok0 + t * tok_per_tile, qbar);
-            const int32_t* table = p.block_table + (size_t)b * p.max_blocks;
-            const long long layer_row0 = (long long)(p.layer0 + l) * p.n_pages;
-            // pool row coordinate of a context tile's two pages; the table is read one tile ahead so that
-            // its latency hides behind the wait for a free slot
-            auto page_rows = [&](int j, int* row) {
-                for (int pg = 0; pg < 2; ++pg) {
-                    const int blk = (tile_begin + j) * 2 + pg;
-                    row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
-                    if (j < n_ctx_tiles && (long long)blk * kPage < seq_len && blk < p.max_blocks) {
-                        const int page = table[blk];
-                        if (page < 0 || page >= p.n_pages)
-                            record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
-                        else
-                            row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
+        }
+        __syncwarp();
+        const int32_t* table = p.block_table + (size_t)b * p.max_blocks;
+        const long long layer_row0 = (long long)(p.layer0 + l) * p.n_pages;
+        // pool row coordinate of a context tile's two pages; the table is read one tile ahead so that
+        // its latency hides behind the wait for a free slot
+        auto page_rows = [&](int j, int* row) {
+            for (int pg = 0; pg < 2; ++pg) {
+                const int blk = (tile_begin + j) * 2 + pg;
+                row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
+                if (j < n_ctx_tiles && (long long)blk * kPage < seq_len && blk < p.max_blocks) {
+                    const int page = table[blk];
+                    if (page < 0 || page >= p.n_pages) {
+                        if (lane == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
+                    } else {
+                        row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
                     }
                 }
-            };
-            int row_next[2];
-            page_rows(0, row_next);
-            for (int j = 0; j < n_tiles; ++j) {
-                const bool is_new = j >= n_ctx_tiles;
-                const int row[2] = {row_next[0], row_next[1]};
-                page_rows(j + 1, row_next);
-                for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
-                    const int use = 2 * j + kv;
-                    const int slot = use % kStages;
-                    const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
-                    if (use >= kStages && !mbar_wait(empty, ((use / kStages) - 1) & 1, abort_flag, p.workspace, 1)) break;
+            }
+        };
+        int row_next[2];
+        page_rows(0, row_next);
+        bool ok = true;
+        uint32_t slot = 0, par = 1;  // ring position of the next use; parity of the release that frees its slot
+        for (int j = 0; j < n_tiles; ++j) {
+            const bool is_new = j >= n_ctx_tiles;
+            const int row[2] = {row_next[0], row_next[1]};
+            page_rows(j + 1, row_next);
+            for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
+                const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
+                if (2 * j + kv >= kStages) ok &= mbar_wait(empty, par, abort_flag, p.workspace, 1);
+                if (lane == 0) {
                     mbar_expect_tx(full, kSlotBytes);
                     const uint32_t dst = kv_smem + slot * kSlotBytes;
                     for (int pg = 0; pg < 2; ++pg)
@@ -245,9 +250,11 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                                 tma_load_2d(d, kv ? &p.tm_vpool : &p.tm_kpool, half * 64, row[pg], full);
                         }
                 }
-                if (*abort_flag) break;
+                __syncwarp();
+                if (++slot == kStages) { slot = 0; par ^= 1; }
             }
         }
+        (void)ok;
     } else if (warp == 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // =========================== MMA issuer ==================================================

@@ -86,3 +86,37 @@ def test_workspace_grows_with_the_request():
     b = B.specpv_workspace_bytes(cfg, 32, 1, 131072, 60)
     c = B.specpv_workspace_bytes(cfg, 32, 4, 131072, 64)
     assert 256 < a < b < c
+
+
+def _rank_main(rank, world, port, q):
+    import torch.distributed as dist
+    import torch
+
+    import bench
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    try:
+        # each replica reports its own device-timed figures; the job's figure is the slowest replica's
+        got = bench.max_over_ranks([10.0 + rank, 5.0 - rank], torch.device("cpu"))
+        q.put((rank, got))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_replica_timings_are_reduced_with_max_over_ranks_gloo():
+    """bench.py --gpus N runs N independent replicas (the path has no exchange step); the only multi-rank
+    logic is the MAX reduction of the timings, exercised here with two gloo ranks on the CPU."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = dict(q.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert results[0] == results[1] == [11.0, 5.0]
