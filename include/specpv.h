@@ -84,6 +84,9 @@ typedef struct {
     float softmax_scale;   /* 0 => 1/sqrt(head_dim) */
     int32_t out_f32;       /* 1 => the attention output O is written as float32 whatever dtype is
                               (the accumulator before the final rounding); 0 => O has type dtype */
+    int32_t select_shared; /* 1 => one block set per (layer, sequence): every KV head keeps the blocks ranked on the
+                              mean of the heads' scores (the paper does not say whether heads select separately);
+                              0 => each KV head selects on its own scores */
 } specpv_config;
 
 typedef struct {
@@ -149,7 +152,9 @@ specpv_status specpv_score_blocks(const specpv_config *cfg, int layer0, int n_la
 /* Section 3.2: the retained block set of every (layer, sequence, KV head): sink blocks, the
  * budget - sink - local best-scored blocks of [sink, nb - local), and the local blocks, written
  * ascending to idx; count[b] = min(nb, budget_blocks).  Ties go to the lower block index, NaN
- * ranks last; the result is a pure function of the float32 scores (bit-exact, deterministic). */
+ * ranks last; the result is a pure function of the float32 scores (bit-exact, deterministic).  With
+ * cfg->select_shared the ranking uses the float32 mean over the KV heads (summed in head order) and all
+ * heads of a layer receive the same list. */
 specpv_status specpv_select_partial_kv(const specpv_config *cfg, int n_layers, const float *scores,
                                        const int32_t *seq_lens, int batch, int max_blocks,
                                        int32_t *idx, int32_t *count, void *workspace,

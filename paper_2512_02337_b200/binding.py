@@ -43,7 +43,7 @@ class Config(ctypes.Structure):
                 ("head_dim", c_int32), ("block_tokens", c_int32), ("dtype", c_int32),
                 ("sink_blocks", c_int32), ("local_blocks", c_int32), ("budget_blocks", c_int32),
                 ("buffer_tokens", c_int32), ("reduce", c_int32), ("score_mode", c_int32),
-                ("softmax_scale", c_float), ("out_f32", c_int32)]
+                ("softmax_scale", c_float), ("out_f32", c_int32), ("select_shared", c_int32)]
 
 
 class PagedKV(ctypes.Structure):
@@ -97,10 +97,10 @@ def _check(status: int, where: str):
 
 
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, dtype, sink_blocks, local_blocks,
-                budget_blocks, buffer_tokens, reduce=REDUCE_MEAN, score_mode=0, softmax_scale=0.0, out_f32=0) -> Config:
+                budget_blocks, buffer_tokens, reduce=REDUCE_MEAN, score_mode=0, softmax_scale=0.0, out_f32=0, select_shared=0) -> Config:
     code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16, "fp32": DTYPE_F32, "bf16": DTYPE_BF16}.get(dtype, dtype)
     return Config(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, code, sink_blocks, local_blocks,
-                  budget_blocks, buffer_tokens, reduce, score_mode, softmax_scale, out_f32)
+                  budget_blocks, buffer_tokens, reduce, score_mode, softmax_scale, out_f32, select_shared)
 
 
 @dataclass

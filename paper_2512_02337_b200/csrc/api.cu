@@ -29,6 +29,7 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     if (cfg->reduce < 0 || cfg->reduce > 2) return SPECPV_ERR_INVALID_ARG;
     if (cfg->score_mode != 0 && cfg->score_mode != 1) return SPECPV_ERR_UNSUPPORTED;
     if (cfg->out_f32 != 0 && cfg->out_f32 != 1) return SPECPV_ERR_INVALID_ARG;
+    if (cfg->select_shared != 0 && cfg->select_shared != 1) return SPECPV_ERR_INVALID_ARG;
     if (!(cfg->softmax_scale >= 0.f) || isinf(cfg->softmax_scale)) return SPECPV_ERR_INVALID_ARG;
     g->n_layers = cfg->n_layers;
     g->Hq = cfg->n_q_heads;
@@ -46,6 +47,7 @@ specpv_status validate_config(const specpv_config* cfg, Geometry* g) {
     g->buffer_tokens = cfg->buffer_tokens;
     g->reduce = cfg->reduce;
     g->score_mode = cfg->score_mode;
+    g->select_shared = cfg->select_shared;
     g->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
     return SPECPV_OK;
 }
@@ -259,6 +261,7 @@ SPECPV_EXPORT specpv_status specpv_select_partial_kv(const specpv_config* cfg, i
     p.scores = scores; p.seq_lens = seq_lens; p.idx = idx; p.count = count; p.batch = batch; p.Hkv = g.Hkv; p.bs = g.bs;
     p.max_blocks = max_blocks; p.sink_blocks = g.sink_blocks; p.local_blocks = g.local_blocks;
     p.budget_blocks = g.budget_blocks;
+    p.share_heads = g.select_shared;
     return launch_select(p, n_layers, reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -217,6 +217,16 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
     const int seq_len = p.seq_lens[b];
     const int nb = min((seq_len + p.bs - 1) / p.bs, p.max_blocks);
     const float* scores = p.scores + (((size_t)l * p.batch + b) * p.Hkv + h) * p.max_blocks;
+    // head-shared selection ranks the blocks on the mean of the layer's KV heads' scores, summed in float32 in
+    // head order (the ranking is a pure function of these bits, the same in every head's CTA)
+    const float* scores_h0 = p.scores + (((size_t)l * p.batch + b) * p.Hkv) * p.max_blocks;
+    const float inv_heads = 1.0f / (float)p.Hkv;
+    auto score_at = [&](int i) {
+        if (!p.share_heads) return scores[i];
+        float acc = 0.f;
+        for (int hh = 0; hh < p.Hkv; ++hh) acc += scores_h0[(size_t)hh * p.max_blocks + i];
+        return acc * inv_heads;
+    };
     int32_t* idx = p.idx + (((size_t)l * p.batch + b) * p.Hkv + h) * p.budget_blocks;
     const int count = min(nb, p.budget_blocks);
     if (l == 0 && h == 0 && tid == 0) p.count[b] = count;
@@ -237,7 +247,7 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
         __syncthreads();
         const uint64_t prefix = s_prefix;
         for (int i = lo + tid; i < hi; i += kSelectThreads) {
-            uint64_t key = select_key(scores[i], i);
+            uint64_t key = select_key(score_at(i), i);
             if ((key & known_mask) == prefix) atomicAdd(&hist[(unsigned)(key >> (8 * pass)) & 255u], 1u);
         }
         __syncthreads();
@@ -263,7 +273,7 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
     __syncthreads();
     for (int base = lo; base < hi; base += kSelectThreads) {
         const int i = base + tid;
-        const bool keep = i < hi && select_key(scores[i], i) >= threshold;
+        const bool keep = i < hi && select_key(score_at(i), i) >= threshold;
         const unsigned ballot = __ballot_sync(0xffffffffu, keep);
         const int warp = tid / 32, lane = tid % 32;
         if (lane == 0) s_warp_counts[warp] = __popc(ballot);

@@ -35,6 +35,7 @@ struct SelectParams {
     int32_t* idx;
     int32_t* count;
     int batch, Hkv, bs, max_blocks, sink_blocks, local_blocks, budget_blocks;
+    int share_heads;  // 1: every KV head of a layer keeps the blocks chosen on the mean of the heads' scores
 };
 
 struct GatherParams {

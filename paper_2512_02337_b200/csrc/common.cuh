@@ -38,7 +38,7 @@ void count_launch(int n = 1);
 struct Geometry {
     int n_layers, Hq, Hkv, G, d, bs, dtype, es;  // es = element size in bytes
     int out_f32, out_es;                          // output element type / size
-    int sink_blocks, local_blocks, budget_blocks, buffer_tokens, reduce, score_mode;
+    int sink_blocks, local_blocks, budget_blocks, buffer_tokens, reduce, score_mode, select_shared;
     float scale;
 };
 

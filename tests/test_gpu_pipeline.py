@@ -13,12 +13,12 @@ from tests import util
 pytestmark = pytest.mark.gpu
 
 
-def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, **over):
+def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, select_shared=0, **over):
     w = wl.make_workload(name, device="cuda", n_layers=n_layers, spare_tokens=256, **over)
     c = w.cfg
     L, Hq, Hkv, d, bs, M = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"]
     batch = w.batch
-    cfg = util.config_for(w, reduce=reduce, score_mode=score_mode)
+    cfg = util.config_for(w, reduce=reduce, score_mode=score_mode, select_shared=select_shared)
     full = util.full_cache(w)
     full.max_seq_len = int(max(c["ctx"])) + 256
     ws = B.new_workspace(cfg, L, batch, full.max_seq_len, M)
@@ -53,7 +53,7 @@ def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, **over):
     B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, out_full, lse_full, ws)
     B.specpv_verify_partial(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, out_part, lse_part, ws)
     if c["dtype"] == "bf16":  # the bfloat16 output is the float32 one, rounded
-        cfg16 = util.config_for(w, reduce=reduce, score_mode=score_mode, out_f32=0)
+        cfg16 = util.config_for(w, reduce=reduce, score_mode=score_mode, select_shared=select_shared, out_f32=0)
         o16f, o16p = torch.zeros_like(out_full, dtype=dt), torch.zeros_like(out_full, dtype=dt)
         B.specpv_verify_full(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, o16f, None, ws)
         B.specpv_verify_partial(cfg16, 0, L, w.q, w.k_new, w.v_new, mask, None, M, partial, o16p, None, ws)
@@ -81,8 +81,12 @@ def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, **over):
             assert np.all(np.isnan(scores_g[l, b, :, nb:]))  # untouched beyond the context
             n_keep = min(nb, cfg.budget_blocks)
             assert count_g[b] == n_keep
-            oidx = np.stack([oracle.select(scores_g[l, b, h, :nb].astype(np.float64), sink, local, cfg.budget_blocks)
-                             for h in range(Hkv)])
+            if select_shared:  # one list per (layer, sequence), ranked on the float32 mean over the heads
+                shared = oracle.head_shared_scores(scores_g[l, b, :, :nb])
+                oidx = np.stack([oracle.select(shared.astype(np.float64), sink, local, cfg.budget_blocks)] * Hkv)
+            else:
+                oidx = np.stack([oracle.select(scores_g[l, b, h, :nb].astype(np.float64), sink, local, cfg.budget_blocks)
+                                 for h in range(Hkv)])
             assert np.array_equal(idx_g[l, b, :, :n_keep], oidx)  # bit-exact given the same float32 scores
             opk, opv = np.zeros_like(pk_g[l]), np.zeros_like(pv_g[l])
             oplen = oracle.gather(kp[l], vp[l], table[b], sl, oidx, opk, opv, first_page=b * ppb)
@@ -129,6 +133,12 @@ def test_channelwise_score_mode_fp32_and_bf16(reduce):
     # score_mode 1: the maximum is taken per channel; selection, gather and partial verification follow from it
     run_pipeline("tiny_fp32", reduce=reduce, score_mode=1)
     run_pipeline("llama_32k", n_layers=1, reduce=reduce, score_mode=1, ctx=[64 * 90 + 3], M=33)
+
+
+def test_head_shared_selection_fp32_and_bf16():
+    # one block set per (layer, sequence): every head gathers and attends the blocks ranked on the heads' mean score
+    run_pipeline("tiny_fp32", select_shared=1)
+    run_pipeline("llama_32k", n_layers=2, select_shared=1, ctx=[64 * 120 + 9], M=25)
 
 
 def test_ragged_batch_shuffled_table_pipeline():

@@ -468,3 +468,17 @@ def test_planted_mistakes_are_caught():
     unmasked, _ = oracle.tree_attention(q, kn, vn, oracle.tree_mask(np.array([-1, 0, 0])), k, v, table, seq_len)
     for wrong in (swapped, negated, unmasked):
         assert np.abs(wrong - out).max() > 1e-3
+
+
+def test_head_shared_scores_is_the_float32_mean_over_heads():
+    rng = np.random.default_rng(5)
+    s = rng.standard_normal((8, 300)).astype(np.float32) * 30
+    got = oracle.head_shared_scores(s)
+    assert got.dtype == np.float32 and got.shape == (300,)
+    np.testing.assert_allclose(got, s.astype(np.float64).mean(axis=0), rtol=4e-7, atol=1e-5)  # float32 rounding only
+    one = oracle.head_shared_scores(s[:1])
+    assert np.array_equal(one, s[0])  # a single head is left as it is
+    # selection on it is ordinary selection: with identical heads the shared list equals every head's own list
+    same = np.repeat(s[:1], 4, axis=0)
+    assert np.array_equal(oracle.select(oracle.head_shared_scores(same).astype(np.float64), 1, 2, 16),
+                          oracle.select(s[0].astype(np.float64), 1, 2, 16))
