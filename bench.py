@@ -282,6 +282,43 @@ def partial_budget_sweep(st, peaks, budgets=(32, 64, 128), iters=10):
     return out
 
 
+def per_layer_graph(st, iters=10):
+    """The same full and partial verification issued the way a model runs them: one call per layer
+    (n_layers = 1), the 32 calls of a pass captured once in a CUDA graph and replayed.  Returns the time of a
+    whole pass (all layers) in microseconds for each."""
+    B, w, cfg, L, M = st["B"], st["w"], st["cfg"], st["L"], st["M"]
+    dev = w.device
+    res = {}
+    for name, cache in (("full_verify_us", st["full"]), ("partial_verify_us", st["partial"])):
+        fn = B.specpv_verify_full if name.startswith("full") else B.specpv_verify_partial
+
+        def one_pass():
+            for l in range(L):
+                fn(cfg, l, 1, w.q[l:l + 1], w.k_new[l:l + 1], w.v_new[l:l + 1], st["mask"], None, M, cache,
+                   st["out"][l:l + 1], st["lse"][l:l + 1], st["ws"])
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(side):
+            one_pass()  # first calls outside the capture (function attributes are set on first use)
+        torch.cuda.current_stream(dev).wait_stream(side)
+        torch.cuda.synchronize(dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_pass()
+        for _ in range(3):
+            graph.replay()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        torch.cuda.synchronize(dev)
+        for a, b in ev:
+            a.record()
+            graph.replay()
+            b.record()
+        torch.cuda.synchronize(dev)
+        res[name] = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+        del graph
+    return res
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -339,6 +376,7 @@ def main():
     ap.add_argument("--budget-blocks", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the per-layer CUDA-graph measurement")
     ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens)")
     args = ap.parse_args()
 
@@ -384,6 +422,9 @@ def main():
     sweep = None
     if not args.no_sweep and rank == 0 and args.budget_blocks is None and c["dtype"] == "bf16":
         sweep = partial_budget_sweep(st, load_peaks())
+    graph_times = None
+    if not args.no_graph and rank == 0 and c["dtype"] == "bf16":
+        graph_times = per_layer_graph(st)
     if rank != 0:
         return 0
 
@@ -428,6 +469,8 @@ def main():
         out["e2e"] = {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     if sweep is not None:
         out["partial_budget_sweep"] = sweep
+    if graph_times is not None:
+        out["per_layer_cuda_graph"] = graph_times
     if not args.no_cpu_baseline and world == 1:
         us, sample, cores = oracle_sample(st)
         out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
