@@ -508,9 +508,15 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     tmem_wait_ld();
                     if (!row_valid) continue;
                     if (!direct) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * kD + c * 32);
+                        // a thread's row is 512 contiguous bytes: 32-byte stores fill whole sectors, half as many
+                        // memory transactions as 16-byte ones for this one-row-per-lane pattern
+                        float* dst = p.part_o + prow * kD + c * 32;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        for (int i = 0; i < 4; ++i)
+                            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 8 * i),
+                                         "r"(v[8 * i]), "r"(v[8 * i + 1]), "r"(v[8 * i + 2]), "r"(v[8 * i + 3]), "r"(v[8 * i + 4]),
+                                         "r"(v[8 * i + 5]), "r"(v[8 * i + 6]), "r"(v[8 * i + 7])
+                                         : "memory");
                     } else if (p.out_f32) {
                         float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_row * kD + c * 32);
 #pragma unroll
