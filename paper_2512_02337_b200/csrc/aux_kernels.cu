@@ -213,6 +213,7 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
     __shared__ int s_remaining;
     __shared__ int s_warp_counts[kSelectThreads / 32];
     __shared__ int s_running;
+    __shared__ int s_round_counts[16 * (kSelectThreads / 32)];  // kept candidates per (round, warp)
     const int h = blockIdx.x, b = blockIdx.y, l = blockIdx.z, tid = threadIdx.x;
     const int seq_len = p.seq_lens[b];
     const int nb = min((seq_len + p.bs - 1) / p.bs, p.max_blocks);
@@ -241,26 +242,50 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
         s_prefix = 0;
         s_remaining = k;
     }
+    // a thread's candidates lo + tid, lo + tid + 256, ...: the first kKeysPerThread keys stay in registers for
+    // all eight passes (enough for 4096 candidate blocks), any further ones are recomputed from the scores
+    constexpr int kKeysPerThread = 16;
+    uint64_t keys[kKeysPerThread];
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        const int i = lo + tid + e * kSelectThreads;
+        keys[e] = i < hi ? select_key(score_at(i), i) : 0ull;  // key 0 cannot occur: the index part of a real key is > 0
+    }
+    const int tail0 = lo + tid + kKeysPerThread * kSelectThreads;
     uint64_t known_mask = 0;
+    const int lane = tid & 31, warp = tid >> 5;
     for (int pass = 7; pass >= 0; --pass) {
         hist[tid] = 0;  // kSelectThreads == 256 bins
         __syncthreads();
         const uint64_t prefix = s_prefix;
-        for (int i = lo + tid; i < hi; i += kSelectThreads) {
-            uint64_t key = select_key(score_at(i), i);
+        const int remaining = s_remaining;
+#pragma unroll
+        for (int e = 0; e < kKeysPerThread; ++e) {
+            const uint64_t key = keys[e];
+            if (key != 0ull && (key & known_mask) == prefix) atomicAdd(&hist[(unsigned)(key >> (8 * pass)) & 255u], 1u);
+        }
+        for (int i = tail0; i < hi; i += kSelectThreads) {
+            const uint64_t key = select_key(score_at(i), i);
             if ((key & known_mask) == prefix) atomicAdd(&hist[(unsigned)(key >> (8 * pass)) & 255u], 1u);
         }
         __syncthreads();
-        if (tid == 0) {
-            int remaining = s_remaining;
-            int bin = 255;
-            unsigned cum = 0;
-            for (; bin > 0; --bin) {
-                if (cum + hist[bin] >= (unsigned)remaining) break;
-                cum += hist[bin];
-            }
-            s_remaining = remaining - (int)cum;
-            s_prefix = prefix | ((uint64_t)bin << (8 * pass));
+        // thread <-> bin: the digit of the k-th largest key is the bin whose suffix count (this bin and all higher
+        // ones) first reaches `remaining`; found in parallel from a block-wide suffix sum
+        const unsigned c = hist[tid];
+        unsigned v = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned up = __shfl_down_sync(0xffffffffu, v, o);
+            if (lane + o < 32) v += up;
+        }
+        if (lane == 0) s_warp_counts[warp] = (int)v;  // count of this warp's 32 bins
+        __syncthreads();
+        unsigned above = 0;
+        for (int w2 = warp + 1; w2 < kSelectThreads / 32; ++w2) above += (unsigned)s_warp_counts[w2];
+        const unsigned suffix = v + above, higher = suffix - c;
+        if (suffix >= (unsigned)remaining && higher < (unsigned)remaining) {  // true for exactly one bin
+            s_remaining = remaining - (int)higher;
+            s_prefix = prefix | ((uint64_t)tid << (8 * pass));
         }
         known_mask |= 0xFFull << (8 * pass);
         __syncthreads();
@@ -269,13 +294,52 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
 
     for (int i = tid; i < p.sink_blocks; i += kSelectThreads) idx[i] = i;
     for (int i = tid; i < p.local_blocks; i += kSelectThreads) idx[p.sink_blocks + k + i] = hi + i;
-    if (tid == 0) s_running = 0;
+    // Ordered compaction of the kept candidates (ascending block index = round e, then thread).  Register part:
+    // one ballot per round, the (round, warp) counts scanned once by warp 0.
+    constexpr int kWarps = kSelectThreads / 32;
+    unsigned ballots[kKeysPerThread];
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        const bool keep = keys[e] != 0ull && keys[e] >= threshold;
+        ballots[e] = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) s_round_counts[e * kWarps + warp] = __popc(ballots[e]);
+    }
     __syncthreads();
-    for (int base = lo; base < hi; base += kSelectThreads) {
+    if (warp == 0) {  // exclusive scan of the 128 counts: four per lane, then across lanes
+        int c4[4], sum = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            c4[u] = s_round_counts[lane * 4 + u];
+            sum += c4[u];
+        }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int run = incl - sum;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            s_round_counts[lane * 4 + u] = run;
+            run += c4[u];
+        }
+        if (lane == 31) s_running = incl;  // kept so far
+    }
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        if ((ballots[e] >> lane) & 1u) {
+            const int offset = s_round_counts[e * kWarps + warp] + __popc(ballots[e] & ((1u << lane) - 1u));
+            if (offset < k) idx[p.sink_blocks + offset] = lo + tid + e * kSelectThreads;
+        }
+    }
+    // candidates beyond the register part (more than 4096 of them): round by round
+    for (int base = lo + kKeysPerThread * kSelectThreads; base < hi; base += kSelectThreads) {
         const int i = base + tid;
         const bool keep = i < hi && select_key(score_at(i), i) >= threshold;
         const unsigned ballot = __ballot_sync(0xffffffffu, keep);
-        const int warp = tid / 32, lane = tid % 32;
+        __syncthreads();  // s_running of the previous round has been read by everyone
         if (lane == 0) s_warp_counts[warp] = __popc(ballot);
         __syncthreads();
         int offset = s_running;
@@ -285,10 +349,9 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(SelectParams p) 
         __syncthreads();
         if (tid == 0) {
             int total = 0;
-            for (int w = 0; w < kSelectThreads / 32; ++w) total += s_warp_counts[w];
+            for (int w = 0; w < kWarps; ++w) total += s_warp_counts[w];
             s_running += total;
         }
-        __syncthreads();
     }
 }
 

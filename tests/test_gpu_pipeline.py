@@ -181,3 +181,33 @@ def test_commit_appends_and_updates_summaries():
     B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax2, kmin2, ws)
     nb = (sl0 + len(path) + bs - 1) // bs
     assert torch.equal(kmax[:, :, :, :nb], kmax2[:, :, :, :nb]) and torch.equal(kmin[:, :, :, :nb], kmin2[:, :, :, :nb])
+
+
+@pytest.mark.parametrize("nb,budget", [(300, 40), (2048, 64), (4099, 128), (9000, 1000)])
+def test_selection_alone_on_synthetic_scores_with_ties_and_nan(nb, budget):
+    """The selection kernel on its own: more candidate blocks than it keeps in registers (nb > 4096), repeated
+    scores (ties go to the lower index), NaN (ranks last), -0 / +0; bit-exact against the oracle."""
+    dev = "cuda"
+    rng = np.random.default_rng(nb)
+    Hkv, L, batch, bs = 3, 2, 2, 64
+    sc = rng.standard_normal((L, batch, Hkv, nb)).astype(np.float32)
+    sc[:, :, 0] = np.round(sc[:, :, 0] * 4) / 4          # many exact ties
+    sc[0, 0, 1, rng.integers(0, nb, size=nb // 7)] = np.nan
+    sc[1, 1, 2, ::5] = -0.0
+    sc[1, 1, 2, 1::5] = 0.0
+    lens = np.array([nb * bs - 3, (nb - 5) * bs], dtype=np.int32)  # ragged last block; a shorter second sequence
+    cfg = B.make_config(L, 8 * Hkv, Hkv, 128, bs, "bf16", 1, 2, budget, 64)
+    scores = torch.from_numpy(sc).to(dev)
+    idx = torch.full((L, batch, Hkv, budget), -7, dtype=torch.int32, device=dev)
+    count = torch.zeros(batch, dtype=torch.int32, device=dev)
+    ws = torch.zeros(4096, dtype=torch.uint8, device=dev)
+    B.specpv_select_partial_kv(cfg, L, scores, torch.from_numpy(lens).to(dev), batch, nb, idx, count, ws)
+    util.sync_status(ws)
+    got = idx.cpu().numpy()
+    for b in range(batch):
+        n = (int(lens[b]) + bs - 1) // bs
+        assert int(count[b]) == min(n, budget)
+        for l in range(L):
+            for h in range(Hkv):
+                want = oracle.select(sc[l, b, h, :n].astype(np.float64), 1, 2, budget)
+                assert np.array_equal(got[l, b, h, :len(want)], want), (l, b, h)
