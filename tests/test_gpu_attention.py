@@ -129,3 +129,46 @@ def test_chain_tree_matches_torch_causal_sdpa():
         q_full.permute(1, 0, 2)[None], k_all.permute(1, 0, 2).repeat_interleave(G, 0)[None],
         v_all.permute(1, 0, 2).repeat_interleave(G, 0)[None], is_causal=True)[0].permute(1, 0, 2)[L:]
     assert (out[0, 0].double().cpu() - want).abs().max() < 1e-5
+
+
+@pytest.mark.parametrize("where", ["late", "early", "middle_twice"])
+def test_large_score_jumps_take_the_general_path(where):
+    """The tensor-core kernel keeps a row's reference maximum across full context tiles and only checks the row sum
+    for overflow; keys whose scores exceed the reference by hundreds of nats (far beyond float32 range of the
+    weights) must send it back over the tile, rescale, and still match the oracle."""
+    dev = "cuda"
+    Hq, Hkv, d, bs, M = 32, 8, 128, 64, 40
+    L_ctx = 64 * 48 + 21
+    g = torch.Generator().manual_seed(17)
+    n_pages = (L_ctx + bs - 1) // bs + 1
+    k_pool = torch.randn((1, n_pages, Hkv, bs, d), generator=g)
+    v_pool = torch.randn((1, n_pages, Hkv, bs, d), generator=g)
+    q = torch.randn((1, 1, M, Hq, d), generator=g)
+    # blocks whose keys are the queries' mean direction, scaled: their logits jump by hundreds of nats
+    direction = q[0, 0].mean(dim=(0, 1))
+    direction = direction / direction.norm()
+    q = q + 8.0 * direction
+    boost = {"late": [(40, 400.0)], "early": [(0, 400.0)], "middle_twice": [(9, 150.0), (30, 500.0)]}[where]
+    for page, scale in boost:
+        k_pool[0, page, :, 5:9] = scale * direction
+    to = lambda t: t.to(torch.bfloat16).to(dev)  # noqa: E731
+    k_pool, v_pool, q = to(k_pool), to(v_pool), to(q)
+    k_new = to(torch.randn((1, 1, M, Hkv, d), generator=g))
+    v_new = to(torch.randn((1, 1, M, Hkv, d), generator=g))
+    rng = np.random.default_rng(3)
+    parents = [wl.make_tree(M, 5, 4, rng)]
+    mask = util.device_masks(parents, M)
+    cfg = B.make_config(1, Hq, Hkv, d, bs, "bf16", 1, 1, 3, bs, out_f32=1)
+    table = torch.arange(n_pages, dtype=torch.int32, device=dev)[None].contiguous()
+    cache = B.Cache(k_pool, v_pool, table, torch.tensor([L_ctx], dtype=torch.int32, device=dev), L_ctx)
+    ws = B.new_workspace(cfg, 1, 1, L_ctx, M)
+    out = torch.zeros((1, 1, M, Hq, d), dtype=torch.float32, device=dev)
+    lse = torch.zeros((1, 1, M, Hq), dtype=torch.float32, device=dev)
+    B.specpv_verify_full(cfg, 0, 1, q, k_new, v_new, mask, None, M, cache, out, lse, ws)
+    util.sync_status(ws)
+    o_out, o_lse = oracle.tree_attention(wl.to_numpy(q[0, 0]), wl.to_numpy(k_new[0, 0]), wl.to_numpy(v_new[0, 0]),
+                                         oracle.tree_mask(parents[0]), wl.to_numpy(k_pool[0]), wl.to_numpy(v_pool[0]),
+                                         table[0].cpu().numpy(), L_ctx)
+    assert np.abs(o_lse).max() > 200  # the jump really is beyond what unscaled float32 weights could hold
+    util.compare(out[0, 0].cpu().numpy(), o_out, "bf16", f"jump {where}")
+    np.testing.assert_allclose(lse[0, 0].cpu().numpy(), o_lse, rtol=2e-5, atol=5e-3)
