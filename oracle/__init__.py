@@ -50,6 +50,10 @@ def _load():
         _lib.oracle_block_scores.restype = None
         _lib.oracle_block_scores_mode.restype = None
         _lib.oracle_tree_attention.restype = None
+        _lib.oracle_step_positions.restype = ctypes.c_int
+        _lib.oracle_linear.restype = None
+        _lib.oracle_rope.restype = None
+        _lib.oracle_qkv_rope.restype = None
     return _lib
 
 
@@ -197,3 +201,49 @@ def select_mode(ctx_len: int, budget_tokens: int, n_partially_verified: int, n_c
                 buffer_tokens: int, partial_initialised: bool) -> int:
     return _load().oracle_select_mode(ctx_len, budget_tokens, n_partially_verified, n_candidates,
                                       buffer_tokens, int(bool(partial_initialised)))
+
+
+# ---- the linear maps either side of the attention (Algorithm 1 "TreeDecode") ------------------------------------
+def step_positions(parents, n_chain: int = 0, base: int = 0) -> np.ndarray:
+    """Sequence positions of a step's rows: chain rows base.., tree node at base + n_chain + depth."""
+    parents = _c(parents, np.int32)
+    pos = np.empty(parents.shape[0] + n_chain, dtype=np.int32)
+    if _load().oracle_step_positions(_p(parents), parents.shape[0], n_chain, base, _p(pos)) != 0:
+        raise ValueError("parents[] is not a tree in topological order")
+    return pos
+
+
+def linear(x, w, residual=None) -> np.ndarray:
+    """y = x w^T (+ residual).  x [T][n_in], w [n_out][n_in] (float32 or bf16 bits) -> [T][n_out] f64."""
+    x, w = _c(x), _c(w)
+    assert _code(x) == _code(w) and x.shape[1] == w.shape[1]
+    if residual is not None:
+        residual = _c(residual)
+        assert _code(residual) == _code(x) and residual.shape == (x.shape[0], w.shape[0])
+    y = np.empty((x.shape[0], w.shape[0]), dtype=np.float64)
+    _load().oracle_linear(_p(x), _p(w), _code(x), x.shape[0], x.shape[1], w.shape[0], _p(residual), _p(y))
+    return y
+
+
+def rope(a, pos, theta: float) -> np.ndarray:
+    """Rotary embedding (half-split pairing) of a [T][H][d] float64 array at positions pos [T]; returns a copy."""
+    a = np.array(a, dtype=np.float64, order="C")
+    T, H, d = a.shape
+    pos = _c(pos, np.int32)
+    assert pos.shape == (T,)
+    _load().oracle_rope(_p(a), T, H, d, _p(pos), ctypes.c_double(theta))
+    return a
+
+
+def qkv_rope(x, w_qkv, Hq: int, Hkv: int, d: int, pos, theta: float):
+    """x [T][hidden], w_qkv [(Hq+2Hkv)d][hidden] -> (q [T][Hq][d], k [T][Hkv][d], v [T][Hkv][d]) f64."""
+    x, w_qkv = _c(x), _c(w_qkv)
+    T, hidden = x.shape
+    assert w_qkv.shape == ((Hq + 2 * Hkv) * d, hidden) and _code(x) == _code(w_qkv)
+    pos = _c(pos, np.int32)
+    q = np.empty((T, Hq, d), dtype=np.float64)
+    k = np.empty((T, Hkv, d), dtype=np.float64)
+    v = np.empty((T, Hkv, d), dtype=np.float64)
+    _load().oracle_qkv_rope(_p(x), _p(w_qkv), _code(x), T, hidden, Hq, Hkv, d, _p(pos), ctypes.c_double(theta),
+                            _p(q), _p(k), _p(v))
+    return q, k, v

@@ -349,3 +349,76 @@ ORACLE_API int oracle_select_mode(int ctx_len, int budget_tokens, int n_partiall
     if (n_partially_verified + n_candidates > buffer_tokens) return 2;
     return 1;
 }
+
+/* ==========================================================================================
+ * The linear maps either side of the verification attention (Algorithm 1 "TreeDecode";
+ * Section 3.3: the refresh pass computes key-value states for the partially verified and the
+ * candidate tokens).  The paper names the step and leaves its arithmetic to the target model;
+ * the readings taken here are those of the LLaMA / Qwen attention block:
+ *   q = x Wq^T, k = x Wk^T, v = x Wv^T  (weights stored [out feature][in feature]),
+ *   rotary position embedding on q and k with the half-split pairing: channel c < d/2 is
+ *   paired with channel c + d/2, angle = position * theta^(-2c/d),
+ *       out[c]       = in[c] cos - in[c + d/2] sin
+ *       out[c + d/2] = in[c + d/2] cos + in[c] sin,
+ *   position of a step token = tokens before the step + its depth in the step (a chain token's
+ *   depth is its index, a tree node's depth counts from the end of the chain),
+ *   o = attn Wo^T (+ residual).
+ * These readings have no pin in the paper ("parity unpinned" by it); the tests pin them to
+ * closed forms and to the properties that define a rotary embedding.
+ * ========================================================================================== */
+
+/* Positions of the step's rows: chain rows base, base+1, ...; tree node i at base + n_chain + depth(i). */
+ORACLE_API int oracle_step_positions(const int32_t *parents, int n_tree, int n_chain, int base, int32_t *pos) {
+    for (int r = 0; r < n_chain; ++r) pos[r] = base + r;
+    for (int i = 0; i < n_tree; ++i) {
+        int p = parents[i];
+        if (i == 0 ? p != -1 : (p < 0 || p >= i)) return -1;
+        int depth = 0;
+        for (int a = i; parents[a] >= 0; a = parents[a]) ++depth;
+        pos[n_chain + i] = base + n_chain + depth;
+    }
+    return 0;
+}
+
+/* y[t][f] = sum_c x[t][c] * w[f][c] (+ residual[t][f]);  x [T][n_in], w [n_out][n_in], y [T][n_out] double. */
+ORACLE_API void oracle_linear(const void *x, const void *w, int dtype, int T, int n_in, int n_out,
+                              const void *residual, double *y) {
+#pragma omp parallel for schedule(static)
+    for (int f = 0; f < n_out; ++f)
+        for (int t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int c = 0; c < n_in; ++c)
+                acc += load_elem(x, dtype, (int64_t)t * n_in + c) * load_elem(w, dtype, (int64_t)f * n_in + c);
+            if (residual) acc += load_elem(residual, dtype, (int64_t)t * n_out + f);
+            y[(int64_t)t * n_out + f] = acc;
+        }
+}
+
+/* Rotary embedding in place on rows [T][H][d] of doubles, row t at position pos[t]. */
+ORACLE_API void oracle_rope(double *a, int T, int H, int d, const int32_t *pos, double theta) {
+    int half = d / 2;
+    for (int t = 0; t < T; ++t)
+        for (int h = 0; h < H; ++h) {
+            double *v = a + ((int64_t)t * H + h) * d;
+            for (int c = 0; c < half; ++c) {
+                double angle = (double)pos[t] * pow(theta, -2.0 * (double)c / (double)d);
+                double cs = cos(angle), sn = sin(angle);
+                double lo = v[c], hi = v[c + half];
+                v[c] = lo * cs - hi * sn;
+                v[c + half] = hi * cs + lo * sn;
+            }
+        }
+}
+
+/* x [T][hidden], w_qkv [(Hq + 2 Hkv) d][hidden] (q heads, then k heads, then v heads) ->
+ * q [T][Hq][d], k [T][Hkv][d] with the rotary embedding, v [T][Hkv][d] without. */
+ORACLE_API void oracle_qkv_rope(const void *x, const void *w_qkv, int dtype, int T, int hidden, int Hq, int Hkv,
+                                int d, const int32_t *pos, double theta, double *q, double *k, double *v) {
+    size_t es = dtype == 0 ? 4 : 2;
+    const char *w = (const char *)w_qkv;
+    oracle_linear(x, w, dtype, T, hidden, Hq * d, NULL, q);
+    oracle_linear(x, w + (size_t)Hq * d * hidden * es, dtype, T, hidden, Hkv * d, NULL, k);
+    oracle_linear(x, w + (size_t)(Hq + Hkv) * d * hidden * es, dtype, T, hidden, Hkv * d, NULL, v);
+    oracle_rope(q, T, Hq, d, pos, theta);
+    oracle_rope(k, T, Hkv, d, pos, theta);
+}

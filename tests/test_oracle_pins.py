@@ -482,3 +482,109 @@ def test_head_shared_scores_is_the_float32_mean_over_heads():
     same = np.repeat(s[:1], 4, axis=0)
     assert np.array_equal(oracle.select(oracle.head_shared_scores(same).astype(np.float64), 1, 2, 16),
                           oracle.select(s[0].astype(np.float64), 1, 2, 16))
+
+
+# ---- the linear maps either side of the attention (Algorithm 1 "TreeDecode") ------------------------------------
+def test_rope_closed_form_pairs_channel_c_with_c_plus_half():
+    """d = 4, theta = 10000, position 1: channel 0 turns by 1 rad into channel 2, channel 1 by 0.01 rad into 3.
+
+    The numbers are cos/sin of 1 and 0.01 typed from tables, so a wrong pairing (neighbouring channels), a wrong
+    sign of the sine or a wrong frequency exponent each miss."""
+    x = np.array([[1, 0, 0, 0], [0, 1, 0, 0], [0, 0, 1, 0]], dtype=np.float32)
+    w = np.tile(np.eye(4, dtype=np.float32), (3, 1))  # q, k and v heads all copy the input
+    q, k, v = oracle.qkv_rope(x, w, 1, 1, 4, [1, 1, 1], 10000.0)
+    want_q = np.array([[0.5403023058681398, 0, 0.8414709848078965, 0],
+                       [0, 0.9999500004166653, 0, 0.009999833334166664],
+                       [-0.8414709848078965, 0, 0.5403023058681398, 0]])
+    np.testing.assert_allclose(q.reshape(3, 4), want_q, atol=1e-15)
+    np.testing.assert_allclose(k.reshape(3, 4), want_q, atol=1e-15)
+    np.testing.assert_array_equal(v.reshape(3, 4), x.astype(np.float64))  # values are never rotated
+
+
+def test_rope_is_a_rotation_that_depends_on_relative_position_only():
+    rng = np.random.default_rng(11)
+    T, H, d = 6, 3, 16
+    a = rng.standard_normal((T, H, d))
+    b = rng.standard_normal((T, H, d))
+    pos = np.array([0, 1, 5, 70000, 131071, 131072], dtype=np.int32)
+    ra, rb = oracle.rope(a, pos, 500000.0), oracle.rope(b, pos, 500000.0)
+    np.testing.assert_array_equal(ra[0], a[0])  # position 0 is the identity
+    np.testing.assert_allclose((ra ** 2).sum(-1), (a ** 2).sum(-1), rtol=1e-12)  # norms kept per head
+    # <R_m a, R_n b> depends on m - n only: shift every position by the same amount
+    for shift in (1, 977, 60000):
+        sa, sb = oracle.rope(a, pos + shift, 500000.0), oracle.rope(b, pos + shift, 500000.0)
+        g0 = np.einsum("thd,uhd->htu", ra, rb)
+        g1 = np.einsum("thd,uhd->htu", sa, sb)
+        np.testing.assert_allclose(g1, g0, atol=1e-8)
+    # and it is not the identity elsewhere
+    assert np.abs(ra[2] - a[2]).max() > 0.1
+
+
+def test_linear_matches_library_matmul_and_is_not_transposed():
+    rng = np.random.default_rng(5)
+    T, n_in, n_out = 7, 48, 20
+    x = rng.standard_normal((T, n_in)).astype(np.float32)
+    w = rng.standard_normal((n_out, n_in)).astype(np.float32)
+    r = rng.standard_normal((T, n_out)).astype(np.float32)
+    np.testing.assert_allclose(oracle.linear(x, w), x.astype(np.float64) @ w.astype(np.float64).T, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear(x, w, r), x.astype(np.float64) @ w.astype(np.float64).T + r, atol=1e-12)
+    # a weight whose row f has a single one at column perm[f] picks input channel perm[f]
+    perm = rng.integers(0, n_in, size=n_out)
+    sel = np.zeros((n_out, n_in), dtype=np.float32)
+    sel[np.arange(n_out), perm] = 1
+    np.testing.assert_array_equal(oracle.linear(x, sel), x[:, perm].astype(np.float64))
+    # bfloat16 inputs are widened exactly
+    xb, wb = bf16_bits(x), bf16_bits(w)
+    np.testing.assert_allclose(oracle.linear(xb, wb), oracle.widen(xb) @ oracle.widen(wb).T, atol=1e-12)
+
+
+def test_qkv_rope_splits_heads_in_q_k_v_order():
+    rng = np.random.default_rng(6)
+    T, hidden, Hq, Hkv, d = 5, 32, 4, 2, 8
+    x = rng.standard_normal((T, hidden)).astype(np.float32)
+    w = rng.standard_normal(((Hq + 2 * Hkv) * d, hidden)).astype(np.float32)
+    pos = np.array([3, 4, 4, 5, 9], dtype=np.int32)
+    q, k, v = oracle.qkv_rope(x, w, Hq, Hkv, d, pos, 10000.0)
+    y = x.astype(np.float64) @ w.astype(np.float64).T
+    np.testing.assert_allclose(v, y[:, (Hq + Hkv) * d:].reshape(T, Hkv, d), atol=1e-12)
+    np.testing.assert_allclose(q, oracle.rope(y[:, :Hq * d].reshape(T, Hq, d), pos, 10000.0), atol=1e-12)
+    np.testing.assert_allclose(k, oracle.rope(y[:, Hq * d:(Hq + Hkv) * d].reshape(T, Hkv, d), pos, 10000.0), atol=1e-12)
+    # at position 0 nothing is rotated
+    q0, k0, _ = oracle.qkv_rope(x, w, Hq, Hkv, d, np.zeros(T, np.int32), 10000.0)
+    np.testing.assert_allclose(q0.reshape(T, -1), y[:, :Hq * d], atol=1e-12)
+    np.testing.assert_allclose(k0.reshape(T, -1), y[:, Hq * d:(Hq + Hkv) * d], atol=1e-12)
+
+
+def test_step_positions_are_base_plus_depth():
+    parents = np.array([-1, 0, 0, 1, 3, 2, 5, 6], dtype=np.int32)
+    # depths by hand: 0, 1, 1, 2, 3, 2, 3, 4
+    np.testing.assert_array_equal(oracle.step_positions(parents, 0, 1000),
+                                  1000 + np.array([0, 1, 1, 2, 3, 2, 3, 4]))
+    np.testing.assert_array_equal(oracle.step_positions(parents, 3, 50),
+                                  np.concatenate([[50, 51, 52], 53 + np.array([0, 1, 1, 2, 3, 2, 3, 4])]))
+    # the depth of a row is also the number of step tokens it sees, minus one
+    m = oracle.tree_mask(parents, 3)
+    seen = np.array([sum(bin(int(wd)).count("1") for wd in row) for row in m])
+    np.testing.assert_array_equal(oracle.step_positions(parents, 3, 0), seen - 1)
+    with pytest.raises(ValueError):
+        oracle.step_positions(np.array([-1, 2, 1], dtype=np.int32))
+
+
+def test_attention_over_own_keys_ignores_where_the_step_starts():
+    """Rotary q and k followed by the tree attention with an empty cache: only position differences enter, so moving
+    the whole step elsewhere in the sequence leaves the output unchanged."""
+    rng = np.random.default_rng(8)
+    T, hidden, Hq, Hkv, d = 9, 24, 4, 2, 16
+    parents = np.array([-1, 0, 0, 1, 1, 2, 4, 4, 6], dtype=np.int32)
+    x = rng.standard_normal((T, hidden)).astype(np.float32)
+    w = (rng.standard_normal(((Hq + 2 * Hkv) * d, hidden)) / np.sqrt(hidden)).astype(np.float32)
+    mask = oracle.tree_mask(parents)
+    empty_k = np.zeros((1, Hkv, 16, d), dtype=np.float32)
+    outs = []
+    for base in (0, 4096, 100000):
+        q, k, v = oracle.qkv_rope(x, w, Hq, Hkv, d, oracle.step_positions(parents, 0, base), 10000.0)
+        out, _ = oracle.tree_attention(q.astype(np.float32), k.astype(np.float32), v.astype(np.float32), mask,
+                                       empty_k, empty_k, np.zeros(1, np.int32), 0)
+        outs.append(out)
+    np.testing.assert_allclose(outs[1], outs[0], atol=2e-5)
+    np.testing.assert_allclose(outs[2], outs[0], atol=2e-5)
