@@ -243,6 +243,48 @@ specpv_status specpv_commit_accepted(const specpv_config *cfg, int layer0, int n
                                      const specpv_paged_kv *dst, void *kmax, void *kmin,
                                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- The linear maps either side of the verification attention -------------------------------
+ * Algorithm 1 "TreeDecode" runs the target model's attention block on the step's tokens, and
+ * Section 3.3 has the refresh pass compute the key-value states of the partially verified and the
+ * candidate tokens.  The paper leaves the block's arithmetic to the target model; these calls
+ * implement the LLaMA / Qwen form: q = x Wq^T, k = x Wk^T, v = x Wv^T with weights stored
+ * [out feature][in feature], a rotary position embedding on q and k that pairs channel c < d/2
+ * with channel c + d/2 (angle = position * theta^(-2c/d)), and o = attn Wo^T (+ residual).
+ * Their outputs are exactly the q / k_new / v_new inputs of the verify calls, and the attention
+ * output (cfg->out_f32 = 0) is the `attn` input of specpv_o_proj.
+ *
+ *   x, attn, residual, y   [n_layers_in_call][batch][M_max][features]   of cfg->dtype
+ *   w_qkv                  [n_layers][(Hq + 2 Hkv) d][hidden]           q heads, then k heads, then v heads
+ *   w_o                    [n_layers][hidden][Hq d]
+ *   cos_sin                [batch][M_max][d/2][2] float32               (cos, sin) of every row's angles
+ * hidden must be a multiple of 16.  bfloat16 with d = 128 and hidden, Hq d multiples of 64 (128 for
+ * the output side of specpv_o_proj) runs on the tensor cores, everything else on a plain kernel.
+ * Rows >= q_lens[b] are computed like any other row (from whatever x holds there); the caller
+ * ignores them. */
+
+/* Positions and angles of a step's rows: row j of sequence b sits at base_pos[b] + depth(j), where
+ * depth(j) = (number of step tokens row j sees under the ancestor-or-self mask) - 1, so that the
+ * partially verified chain of a refresh counts on from base_pos[b] and the tree from the chain's end.
+ * base_pos (device [batch]) = tokens of the sequence in front of the step (full-cache length in a full
+ * or refresh step, full-cache length + partially verified tokens in a partial step).  The angles are
+ * formed in double precision and rounded once to float32.  One table serves every layer of the step. */
+specpv_status specpv_rope_table(const specpv_config *cfg, const uint64_t *tree_mask, const int32_t *q_lens,
+                                const int32_t *base_pos, int batch, int M_max, double rope_theta,
+                                float *cos_sin, void *stream);
+
+/* q, k_new (rotated) and v_new (not rotated) of the step's tokens for layers [layer0, layer0 + n_layers)
+ * of w_qkv; x, q, k_new, v_new are indexed by layer-in-call.  Needs no more workspace than the verify
+ * calls (specpv_workspace_bytes); a smaller workspace only costs speed. */
+specpv_status specpv_qkv_rope(const specpv_config *cfg, int layer0, int n_layers, const void *x, int hidden,
+                              const void *w_qkv, const float *cos_sin, int batch, int M_max, void *q,
+                              void *k_new, void *v_new, void *workspace, size_t workspace_bytes, void *stream);
+
+/* y = attn Wo^T (+ residual if not NULL) for the same rows; attn is the attention output
+ * [..][Hq][d] read as [..][Hq d]. */
+specpv_status specpv_o_proj(const specpv_config *cfg, int layer0, int n_layers, const void *attn,
+                            const void *w_o, int hidden, const void *residual, int batch, int M_max, void *y,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ EXPORTS = [
     "specpv_select_mode", "specpv_update_block_summaries", "specpv_score_blocks",
     "specpv_select_partial_kv", "specpv_refresh_partial", "specpv_verify_partial",
     "specpv_verify_full", "specpv_verify_host", "specpv_commit_accepted", "specpv_verify_partial_static",
+    "specpv_rope_table", "specpv_qkv_rope", "specpv_o_proj",
 ]
 
 
@@ -246,3 +247,24 @@ def specpv_commit_accepted(cfg, layer0, n_layers, k_new, v_new, M_max, accepted,
                                         _ptr(accepted), _ptr(n_accepted), A_max, ctypes.byref(d), _ptr(kmax),
                                         _ptr(kmin), _ptr(workspace), c_size_t(workspace.numel()), _stream(stream)),
            "specpv_commit_accepted")
+
+
+# ---- the linear maps either side of the attention ---------------------------------------------------------------
+def specpv_rope_table(cfg, tree_mask, q_lens, base_pos, batch, M_max, rope_theta, cos_sin, stream=None):
+    _check(lib().specpv_rope_table(ctypes.byref(cfg), _ptr(tree_mask), _ptr(q_lens), _ptr(base_pos), batch, M_max,
+                                   ctypes.c_double(rope_theta), _ptr(cos_sin), _stream(stream)),
+           "specpv_rope_table")
+
+
+def specpv_qkv_rope(cfg, layer0, n_layers, x, hidden, w_qkv, cos_sin, batch, M_max, q, k_new, v_new, workspace,
+                    stream=None):
+    _check(lib().specpv_qkv_rope(ctypes.byref(cfg), layer0, n_layers, _ptr(x), hidden, _ptr(w_qkv), _ptr(cos_sin),
+                                 batch, M_max, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(workspace),
+                                 c_size_t(workspace.numel()), _stream(stream)),
+           "specpv_qkv_rope")
+
+
+def specpv_o_proj(cfg, layer0, n_layers, attn, w_o, hidden, residual, batch, M_max, y, workspace, stream=None):
+    _check(lib().specpv_o_proj(ctypes.byref(cfg), layer0, n_layers, _ptr(attn), _ptr(w_o), hidden, _ptr(residual),
+                               batch, M_max, _ptr(y), _ptr(workspace), c_size_t(workspace.numel()), _stream(stream)),
+           "specpv_o_proj")

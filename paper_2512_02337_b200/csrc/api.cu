@@ -6,6 +6,7 @@
 
 #include "aux_kernels.cuh"
 #include "common.cuh"
+#include "proj.cuh"
 
 #define SPECPV_EXPORT extern "C" __attribute__((visibility("default")))
 
@@ -454,4 +455,74 @@ SPECPV_EXPORT specpv_status specpv_commit_accepted(const specpv_config* cfg, int
         return launch_commit_lens(const_cast<int32_t*>(dst->seq_lens), n_accepted, dst->batch, A_max,
                                   dst->max_blocks * g.bs, s);
     return SPECPV_OK;
+}
+
+// ---- the linear maps either side of the attention --------------------------------------------------------------
+SPECPV_EXPORT specpv_status specpv_rope_table(const specpv_config* cfg, const uint64_t* tree_mask, const int32_t* q_lens,
+                                              const int32_t* base_pos, int batch, int M_max, double rope_theta,
+                                              float* cos_sin, void* stream) {
+    Geometry g;
+    specpv_status st = validate_config(cfg, &g);
+    if (st != SPECPV_OK) return st;
+    if (!tree_mask || !base_pos || !cos_sin || !aligned16(cos_sin)) return SPECPV_ERR_INVALID_ARG;
+    if (batch <= 0 || M_max <= 0 || !(rope_theta > 1.0) || isinf(rope_theta)) return SPECPV_ERR_INVALID_ARG;
+    if (M_max > kMaxQTokens) return SPECPV_ERR_CAPACITY;
+    return launch_rope_table(tree_mask, q_lens, base_pos, batch, M_max, g.d, rope_theta, cos_sin,
+                             reinterpret_cast<cudaStream_t>(stream));
+}
+
+static specpv_status proj_dispatch(ProjArgs& a, const Geometry& g, int layer0, int n_layers, int batch, int M_max,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || !aligned16(workspace) || workspace_bytes < kStatusBytes) return SPECPV_ERR_INVALID_ARG;
+    if (layer0 < 0 || n_layers <= 0 || layer0 + n_layers > g.n_layers || batch <= 0 || M_max <= 0)
+        return SPECPV_ERR_INVALID_ARG;
+    if ((int64_t)batch * M_max > (int64_t)1 << 24) return SPECPV_ERR_CAPACITY;
+    a.dtype = g.dtype;
+    a.layer0 = layer0; a.n_layers_call = n_layers; a.n_layers_total = g.n_layers;
+    a.tokens = batch * M_max;
+    a.workspace = workspace;
+    a.scratch_off = kStatusBytes;
+    a.scratch_bytes = workspace_bytes - kStatusBytes;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (proj_tc_supported(a)) return launch_proj_tc(a, s);
+    return launch_proj_simt(a, s);
+}
+
+SPECPV_EXPORT specpv_status specpv_qkv_rope(const specpv_config* cfg, int layer0, int n_layers, const void* x, int hidden,
+                                            const void* w_qkv, const float* cos_sin, int batch, int M_max, void* q,
+                                            void* k_new, void* v_new, void* workspace, size_t workspace_bytes,
+                                            void* stream) {
+    Geometry g;
+    specpv_status st = validate_config(cfg, &g);
+    if (st != SPECPV_OK) return st;
+    if (!x || !w_qkv || !cos_sin || !q || !k_new || !v_new) return SPECPV_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(cos_sin) || !aligned16(q) || !aligned16(k_new) || !aligned16(v_new))
+        return SPECPV_ERR_INVALID_ARG;
+    if (hidden <= 0 || hidden % 16 != 0) return SPECPV_ERR_SHAPE;
+    ProjArgs a{};
+    a.x = x; a.w = w_qkv; a.cos_sin = cos_sin; a.residual = nullptr;
+    a.n_in = hidden; a.n_out = (g.Hq + 2 * g.Hkv) * g.d; a.tile = g.d;
+    a.n_seg = 3;
+    a.seg[0] = ProjSegment{q, 0, g.Hq * g.d, 1};
+    a.seg[1] = ProjSegment{k_new, g.Hq, g.Hkv * g.d, 1};
+    a.seg[2] = ProjSegment{v_new, g.Hq + g.Hkv, g.Hkv * g.d, 0};
+    return proj_dispatch(a, g, layer0, n_layers, batch, M_max, workspace, workspace_bytes, stream);
+}
+
+SPECPV_EXPORT specpv_status specpv_o_proj(const specpv_config* cfg, int layer0, int n_layers, const void* attn,
+                                          const void* w_o, int hidden, const void* residual, int batch, int M_max, void* y,
+                                          void* workspace, size_t workspace_bytes, void* stream) {
+    Geometry g;
+    specpv_status st = validate_config(cfg, &g);
+    if (st != SPECPV_OK) return st;
+    if (!attn || !w_o || !y) return SPECPV_ERR_INVALID_ARG;
+    if (!aligned16(attn) || !aligned16(w_o) || !aligned16(y) || (residual && !aligned16(residual)))
+        return SPECPV_ERR_INVALID_ARG;
+    if (hidden <= 0 || hidden % 16 != 0) return SPECPV_ERR_SHAPE;
+    ProjArgs a{};
+    a.x = attn; a.w = w_o; a.cos_sin = nullptr; a.residual = residual;
+    a.n_in = g.Hq * g.d; a.n_out = hidden; a.tile = hidden % 128 == 0 ? 128 : 16;
+    a.n_seg = 1;
+    a.seg[0] = ProjSegment{y, 0, hidden, 0};
+    return proj_dispatch(a, g, layer0, n_layers, batch, M_max, workspace, workspace_bytes, stream);
 }

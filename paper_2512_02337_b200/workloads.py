@@ -205,3 +205,52 @@ def make_workload(name: str, device="cpu", n_layers: int | None = None, spare_to
                     k_pool=k_pool, v_pool=v_pool, block_table=table_t,
                     seq_lens=torch.tensor(ctx, dtype=torch.int32, device=device),
                     q=q, k_new=k_new, v_new=v_new, parents=parents)
+
+
+# hidden size and rotary base of the attention block each config's head geometry comes from
+# (LLaMA-3.1-8B: 4096 / 5e5, Qwen3-8B: 4096 / 1e6; the tiny config: Hq * d / 1e4)
+BLOCK_SHAPES = {
+    "tiny_fp32": (512, 1.0e4),
+    "llama_32k": (4096, 5.0e5),
+    "llama_128k": (4096, 5.0e5),
+    "qwen3_64k_loop": (4096, 1.0e6),
+    "stress_b4": (4096, 5.0e5),
+}
+
+
+@dataclass
+class BlockWeights:
+    """Synthetic inputs of the linear maps either side of the attention (random-init weights)."""
+    hidden: int
+    rope_theta: float
+    x: torch.Tensor         # [n_layers][batch][M][hidden]   hidden states entering the block
+    residual: torch.Tensor  # [n_layers][batch][M][hidden]
+    w_qkv: torch.Tensor     # [n_layers][(Hq + 2 Hkv) d][hidden]
+    w_o: torch.Tensor       # [n_layers][hidden][Hq d]
+
+
+def make_block_weights(name: str, device="cpu", n_layers: int | None = None, M: int | None = None,
+                       hidden: int | None = None, **overrides) -> BlockWeights:
+    """x ~ N(0, 1); weights ~ N(0, 1 / fan-in) so that q, k, v and the block output stay near unit scale."""
+    cfg = dict(CONFIGS[name])
+    cfg.update(overrides)
+    L = cfg["n_layers"] if n_layers is None else n_layers
+    M = cfg["M"] if M is None else M
+    hid, theta = BLOCK_SHAPES[name]
+    hid = hid if hidden is None else hidden
+    Hq, Hkv, d = cfg["Hq"], cfg["Hkv"], cfg["d"]
+    batch = len(cfg["ctx"])
+    dt = torch_dtype(cfg["dtype"])
+    device = torch.device(device)
+    seed = BASE_SEED + cfg["index"]
+    x = torch.empty((L, batch, M, hid), dtype=dt, device=device)
+    res = torch.empty_like(x)
+    w_qkv = torch.empty((L, (Hq + 2 * Hkv) * d, hid), dtype=dt, device=device)
+    w_o = torch.empty((L, hid, Hq * d), dtype=dt, device=device)
+    for layer in range(L):
+        g = _gen(seed, 2, layer, device)
+        x[layer] = torch.randn((batch, M, hid), generator=g, device=device).to(dt)
+        res[layer] = torch.randn((batch, M, hid), generator=g, device=device).to(dt)
+        w_qkv[layer] = (torch.randn(((Hq + 2 * Hkv) * d, hid), generator=g, device=device) / hid ** 0.5).to(dt)
+        w_o[layer] = (torch.randn((hid, Hq * d), generator=g, device=device) / (Hq * d) ** 0.5).to(dt)
+    return BlockWeights(hidden=hid, rope_theta=theta, x=x, residual=res, w_qkv=w_qkv, w_o=w_o)
