@@ -319,6 +319,78 @@ def per_layer_graph(st, iters=10):
     return res
 
 
+def attention_block(st, peaks, iters=10):
+    """The linear maps either side of the attention (QKV projection with rotary embedding, output projection with
+    residual) on random-init weights of the model's hidden size: each alone as one layer-batched launch (all
+    layers' weights streamed once, more than L2), and the whole block (QKV -> partial verification -> output
+    projection) issued per layer and replayed from a CUDA graph.  `frac` is against the HBM time of the weights
+    plus the step tensors each launch has to move."""
+    B, w, cfg, L, M, batch = st["B"], st["w"], st["cfg"], st["L"], st["M"], st["batch"]
+    c = w.cfg
+    Hq, Hkv, d = c["Hq"], c["Hkv"], c["d"]
+    dev = w.device
+    bw = wl.make_block_weights(w.name, device=dev, n_layers=L)
+    hid = bw.hidden
+    base = (w.seq_lens + 0).to(torch.int32)
+    cos_sin = torch.zeros((batch, M, d // 2, 2), dtype=torch.float32, device=dev)
+    B.specpv_rope_table(cfg, st["mask"], None, base, batch, M, bw.rope_theta, cos_sin)
+    q, k_new, v_new = torch.empty_like(w.q), torch.empty_like(w.k_new), torch.empty_like(w.v_new)
+    y = torch.empty_like(bw.x)
+    ws = st["ws"]
+    es = 2
+    calls = {
+        "qkv_rope": (lambda: B.specpv_qkv_rope(cfg, 0, L, bw.x, hid, bw.w_qkv, cos_sin, batch, M, q, k_new, v_new, ws),
+                     L * ((Hq + 2 * Hkv) * d * hid + batch * M * (hid + (Hq + 2 * Hkv) * d)) * es),
+        "o_proj": (lambda: B.specpv_o_proj(cfg, 0, L, st["out"], bw.w_o, hid, bw.residual, batch, M, y, ws),
+                   L * (hid * Hq * d + batch * M * (Hq * d + 2 * hid)) * es),
+    }
+    res = {"hidden": hid}
+    for name, (call, nbytes) in calls.items():
+        for _ in range(3):
+            call()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        torch.cuda.synchronize(dev)
+        for a, b in ev:
+            a.record()
+            call()
+            b.record()
+        torch.cuda.synchronize(dev)
+        us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+        res[name] = {"us": us, "gbs": nbytes / (us * 1e-6) / 1e9, "frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6)}
+
+    def one_pass():
+        for l in range(L):
+            B.specpv_qkv_rope(cfg, l, 1, bw.x[l:l + 1], hid, bw.w_qkv, cos_sin, batch, M, q[l:l + 1], k_new[l:l + 1],
+                              v_new[l:l + 1], ws)
+            B.specpv_verify_partial(cfg, l, 1, q[l:l + 1], k_new[l:l + 1], v_new[l:l + 1], st["mask"], None, M,
+                                    st["partial"], st["out"][l:l + 1], st["lse"][l:l + 1], ws)
+            B.specpv_o_proj(cfg, l, 1, st["out"][l:l + 1], bw.w_o, hid, bw.residual[l:l + 1], batch, M, y[l:l + 1], ws)
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(side):
+        one_pass()
+    torch.cuda.current_stream(dev).wait_stream(side)
+    torch.cuda.synchronize(dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one_pass()
+    for _ in range(3):
+        graph.replay()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    torch.cuda.synchronize(dev)
+    for a, b in ev:
+        a.record()
+        graph.replay()
+        b.record()
+    torch.cuda.synchronize(dev)
+    us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+    block_bytes = calls["qkv_rope"][1] + calls["o_proj"][1] + int(st["plens"].sum()) * L * Hkv * 2 * d * es
+    res["per_layer_block_graph"] = {"us": us, "bound_us": block_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                                    "frac": block_bytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6)}
+    del graph
+    return res
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -377,6 +449,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the per-layer CUDA-graph measurement")
+    ap.add_argument("--no-block", action="store_true",
+                    help="skip the QKV / output projection measurement (the linear maps either side of the attention)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens)")
     args = ap.parse_args()
 
@@ -425,6 +499,9 @@ def main():
     graph_times = None
     if not args.no_graph and rank == 0 and c["dtype"] == "bf16":
         graph_times = per_layer_graph(st)
+    block = None
+    if not args.no_block and rank == 0 and c["dtype"] == "bf16":
+        block = attention_block(st, load_peaks())
     if rank != 0:
         return 0
 
@@ -471,6 +548,8 @@ def main():
         out["partial_budget_sweep"] = sweep
     if graph_times is not None:
         out["per_layer_cuda_graph"] = graph_times
+    if block is not None:
+        out["attention_block"] = block
     if not args.no_cpu_baseline and world == 1:
         us, sample, cores = oracle_sample(st)
         out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}

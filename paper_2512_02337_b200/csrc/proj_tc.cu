@@ -26,6 +26,10 @@ constexpr int kWTileBytes = kFeatTile * 128;  // 128 features x 64 input feature
 constexpr int kProjDataBytes = 192 * 1024;
 constexpr int kProjSmem = 1024 + kProjDataBytes;
 constexpr int kProjMaxStages = 8;
+#ifndef PROJ_ISSUE_GROUP
+#define PROJ_ISSUE_GROUP 2
+#endif
+constexpr int kIssueGroup = PROJ_ISSUE_GROUP;  // stages whose copies are issued together
 constexpr int kMaxTokTile = 256;           // rows per CTA (accumulator columns)
 
 struct ProjTcParams {
@@ -36,7 +40,7 @@ struct ProjTcParams {
     float* partials;
     void* workspace;
     ProjSegment seg[3];
-    int n_seg, layer0, n_tiles, n_out, tokens, n_pad, ksteps, splits, stages;
+    int n_seg, layer0, n_tiles, n_out, tokens, n_pad, ksteps, splits, stages, group;
 };
 
 struct __align__(8) ProjBarriers {
@@ -54,7 +58,7 @@ __device__ __forceinline__ void proj_finish(const ProjTcParams& p, int tile, int
         if (tile >= p.seg[i].first_tile) s = i;
     const ProjSegment& sg = p.seg[s];
     if (sg.rope) {
-        const float4 cs = *reinterpret_cast<const float4*>(p.cos_sin + ((size_t)tok * 64 + 2 * j) * 2);  // cos, sin, cos, sin
+        const float4 cs = __ldg(reinterpret_cast<const float4*>(p.cos_sin + ((size_t)tok * 64 + 2 * j) * 2));  // cos, sin, cos, sin
         const float2 rl = make_float2(lo.x * cs.x - hi.x * cs.y, lo.y * cs.z - hi.y * cs.w);
         const float2 rh = make_float2(hi.x * cs.x + lo.x * cs.y, hi.y * cs.z + lo.y * cs.w);
         lo = rl;
@@ -62,10 +66,10 @@ __device__ __forceinline__ void proj_finish(const ProjTcParams& p, int tile, int
     }
     const size_t off = ((size_t)l * p.tokens + tok) * sg.row_stride + (size_t)(tile - sg.first_tile) * kFeatTile + 2 * j;
     if (p.residual && s == 0) {
-        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(p.residual + off);
-        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(p.residual + off + 64);
-        lo.x += __bfloat162float(a.x); lo.y += __bfloat162float(a.y);
-        hi.x += __bfloat162float(b.x); hi.y += __bfloat162float(b.y);
+        const uint32_t a = __ldg(reinterpret_cast<const uint32_t*>(p.residual + off));
+        const uint32_t b = __ldg(reinterpret_cast<const uint32_t*>(p.residual + off + 64));
+        lo.x += __uint_as_float(a << 16); lo.y += __uint_as_float(a & 0xFFFF0000u);
+        hi.x += __uint_as_float(b << 16); hi.y += __uint_as_float(b & 0xFFFF0000u);
     }
     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(sg.base) + off;
     *reinterpret_cast<uint32_t*>(dst) = pack_bf16(lo.x, lo.y);
@@ -77,7 +81,7 @@ __device__ __forceinline__ size_t partial_base(const ProjTcParams& p, int l, int
     return (unit * p.splits + split) * (size_t)p.n_pad * kFeatTile;
 }
 
-__global__ void __launch_bounds__(kProjThreads, 1) proj_tc_kernel(const __grid_constant__ ProjTcParams p) {
+__global__ void __launch_bounds__(kProjThreads, 2) proj_tc_kernel(const __grid_constant__ ProjTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ ProjBarriers bars;
@@ -118,16 +122,23 @@ __global__ void __launch_bounds__(kProjThreads, 1) proj_tc_kernel(const __grid_c
         const int w_row = (p.layer0 + l) * p.n_out + tile * kFeatTile;
         const int x_row = l * p.tokens + tok0;
         bool ok = true;
-        for (int i = 0; i < n_k; ++i) {
-            const int slot = i % p.stages;
-            if (i >= p.stages)
-                ok &= mbar_wait(smem_u32(&bars.empty[slot]), ((i / p.stages) - 1) & 1, abort_flag, p.workspace, 30);
+        // The copies of p.group consecutive stages are issued together: a weight row is 128 contiguous bytes
+        // per stage, and DRAM serves the same row's neighbouring chunks far better when they are asked for at
+        // nearly the same time than one stage apart.
+        for (int i0 = 0; i0 < n_k; i0 += p.group) {
+            const int i1 = min(i0 + p.group, n_k);
+            for (int i = i0; i < i1; ++i)
+                if (i >= p.stages)
+                    ok &= mbar_wait(smem_u32(&bars.empty[i % p.stages]), ((i / p.stages) - 1) & 1, abort_flag, p.workspace, 30);
             if (lane == 0 && ok) {
-                const uint32_t full = smem_u32(&bars.full[slot]);
-                const uint32_t dst = data + slot * stage_bytes;
-                mbar_expect_tx(full, stage_bytes);
-                tma_load_2d(dst, &p.tm_w, (kb + i) * 64, w_row, full);
-                tma_load_2d(dst + kWTileBytes, &p.tm_x, (kb + i) * 64, x_row, full);
+                for (int i = i0; i < i1; ++i) {
+                    const int slot = i % p.stages;
+                    const uint32_t full = smem_u32(&bars.full[slot]);
+                    const uint32_t dst = data + slot * stage_bytes;
+                    mbar_expect_tx(full, stage_bytes);
+                    tma_load_2d(dst, &p.tm_w, (kb + i) * 64, w_row, full);
+                    tma_load_2d(dst + kWTileBytes, &p.tm_x, (kb + i) * 64, x_row, full);
+                }
             }
             __syncwarp();
         }
@@ -173,6 +184,7 @@ __global__ void __launch_bounds__(kProjThreads, 1) proj_tc_kernel(const __grid_c
         if (ok) {
             const int et = threadIdx.x - 64, j = et & 31;
             float* part = p.splits > 1 ? p.partials + partial_base(p, l, chunk, gridDim.y, tile, split) : nullptr;
+#pragma unroll 4
             for (int t = et >> 5; t < valid; t += 4) {
                 const float2 lo = *reinterpret_cast<const float2*>(stage + t * kFeatTile + 2 * j);
                 const float2 hi = *reinterpret_cast<const float2*>(stage + t * kFeatTile + 64 + 2 * j);
@@ -194,23 +206,30 @@ __global__ void __launch_bounds__(kProjThreads, 1) proj_tc_kernel(const __grid_c
     }
 }
 
-// Adds the partial sums of a tile's input-feature ranges in range order and finishes the rows.
-__global__ void __launch_bounds__(128) proj_reduce_kernel(const __grid_constant__ ProjTcParams p) {
-    const int tile = blockIdx.x, chunk = blockIdx.y, l = blockIdx.z;
+// Adds the partial sums of a tile's input-feature ranges in range order and finishes the rows: a CTA takes four rows
+// of one tile, a thread one row's channels (2j, 2j+1, 64+2j, 64+2j+1), so that all its loads are in flight together.
+__global__ void __launch_bounds__(128) proj_reduce_kernel(const __grid_constant__ ProjTcParams p, int n_chunks) {
+    const int tile = blockIdx.x, l = blockIdx.z / n_chunks, chunk = blockIdx.z % n_chunks;
     const int tok0 = chunk * kMaxTokTile;
     const int valid = min(p.n_pad, p.tokens - tok0);
-    const int j = threadIdx.x & 31;
-    const float* part = p.partials + partial_base(p, l, chunk, gridDim.y, tile, 0);
+    const int j = threadIdx.x & 31, t = blockIdx.y * 4 + (threadIdx.x >> 5);
+    if (t >= valid) return;
+    const float* part = p.partials + partial_base(p, l, chunk, n_chunks, tile, 0) + (size_t)t * kFeatTile + 2 * j;
     const size_t split_stride = (size_t)p.n_pad * kFeatTile;
-    for (int t = threadIdx.x >> 5; t < valid; t += 4) {
-        float2 lo = make_float2(0.f, 0.f), hi = lo;
-        for (int s = 0; s < p.splits; ++s) {
-            const float2 a = *reinterpret_cast<const float2*>(part + s * split_stride + (size_t)t * kFeatTile + 2 * j);
-            const float2 b = *reinterpret_cast<const float2*>(part + s * split_stride + (size_t)t * kFeatTile + 64 + 2 * j);
-            lo.x += a.x; lo.y += a.y; hi.x += b.x; hi.y += b.y;
+    float2 a[8], b[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+        if (s < p.splits) {
+            a[s] = __ldg(reinterpret_cast<const float2*>(part + s * split_stride));
+            b[s] = __ldg(reinterpret_cast<const float2*>(part + s * split_stride + 64));
         }
-        proj_finish(p, tile, l, tok0 + t, j, lo, hi);
-    }
+    float2 lo = make_float2(0.f, 0.f), hi = lo;
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+        if (s < p.splits) {
+            lo.x += a[s].x; lo.y += a[s].y; hi.x += b[s].x; hi.y += b[s].y;
+        }
+    proj_finish(p, tile, l, tok0 + t, j, lo, hi);
 }
 
 // ---- plain kernel: any dtype / head size ---------------------------------------------------------------------
@@ -322,8 +341,12 @@ specpv_status launch_proj_tc(const ProjArgs& a, cudaStream_t stream) {
     p.layer0 = a.layer0; p.n_tiles = a.n_out / kFeatTile; p.n_out = a.n_out; p.tokens = a.tokens;
     p.ksteps = a.n_in / 64;
     const int stage_bytes = kWTileBytes + p.n_pad * 128;
-    p.stages = kProjDataBytes / stage_bytes;
+    // up to 128 rows the ring and the epilogue's staging tile fit in half the shared memory, and two CTAs per SM
+    // cover each other's start and epilogue
+    const int ring_bytes = p.n_pad <= 128 ? kProjDataBytes / 2 : kProjDataBytes;
+    p.stages = ring_bytes / stage_bytes;
     if (p.stages > kProjMaxStages) p.stages = kProjMaxStages;
+    p.group = kIssueGroup <= p.stages / 2 ? kIssueGroup : (p.stages / 2 > 0 ? p.stages / 2 : 1);
     // enough CTAs to keep every SM streaming weights: split the input features while the tiles alone cannot
     const long long units = (long long)a.n_layers_call * n_chunks * p.n_tiles;
     int splits = 1;
@@ -337,11 +360,11 @@ specpv_status launch_proj_tc(const ProjArgs& a, cudaStream_t stream) {
     p.splits = splits;
     p.partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + a.scratch_off);
     dim3 grid(p.n_tiles * splits, n_chunks, a.n_layers_call);
-    proj_tc_kernel<<<grid, kProjThreads, kProjSmem, stream>>>(p);
+    proj_tc_kernel<<<grid, kProjThreads, 1024 + ring_bytes, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
     if (splits > 1) {
-        proj_reduce_kernel<<<dim3(p.n_tiles, n_chunks, a.n_layers_call), 128, 0, stream>>>(p);
+        proj_reduce_kernel<<<dim3(p.n_tiles, (p.n_pad + 3) / 4, a.n_layers_call * n_chunks), 128, 0, stream>>>(p, n_chunks);
         if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
         count_launch();
     }
