@@ -343,15 +343,17 @@ specpv_status launch_proj_tc(const ProjArgs& a, cudaStream_t stream) {
     const int stage_bytes = kWTileBytes + p.n_pad * 128;
     // up to 128 rows the ring and the epilogue's staging tile fit in half the shared memory, and two CTAs per SM
     // cover each other's start and epilogue
-    const int ring_bytes = p.n_pad <= 128 ? kProjDataBytes / 2 : kProjDataBytes;
+    const bool small_ring = p.n_pad <= 128;
+    const int ring_bytes = small_ring ? kProjDataBytes / 2 : kProjDataBytes;
     p.stages = ring_bytes / stage_bytes;
     if (p.stages > kProjMaxStages) p.stages = kProjMaxStages;
     p.group = kIssueGroup <= p.stages / 2 ? kIssueGroup : (p.stages / 2 > 0 ? p.stages / 2 : 1);
-    // enough CTAs to keep every SM streaming weights: split the input features while the tiles alone cannot
+    // enough CTAs to fill every SM's slots: split the input features while the tiles alone cannot
     const long long units = (long long)a.n_layers_call * n_chunks * p.n_tiles;
+    const int slots = small_ring ? 2 * 148 : 148;
     int splits = 1;
     if (units < 120) {
-        splits = (int)(148 / units);
+        splits = (int)(slots / units);
         if (splits > 8) splits = 8;
         if (splits > p.ksteps) splits = p.ksteps;
         const size_t per_split = (size_t)units * p.n_pad * kFeatTile * sizeof(float);

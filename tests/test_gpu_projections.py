@@ -66,8 +66,8 @@ CASES = [
     # dtype, Hq, Hkv, d, hidden, batch, M, n_layers (pool), layer0, n_call
     ("fp32", 8, 2, 64, 512, 1, 16, 1, 0, 1),        # plain path, the tiny config's geometry
     ("bf16", 4, 2, 64, 192, 2, 9, 2, 1, 1),         # plain path in bfloat16, second layer of the pool
-    ("bf16", 32, 8, 128, 4096, 1, 60, 1, 0, 1),     # tensor cores, one layer: three input ranges per tile
-    ("bf16", 8, 2, 128, 448, 1, 37, 3, 1, 2),       # seven 64-wide input steps over six ranges, layers 1-2 of 3
+    ("bf16", 32, 8, 128, 4096, 1, 60, 1, 0, 1),     # tensor cores, one layer: six input ranges per tile
+    ("bf16", 8, 2, 128, 448, 1, 37, 3, 1, 2),       # seven 64-wide input steps over seven ranges, layers 1-2 of 3
     ("bf16", 8, 4, 128, 1024, 4, 64, 10, 0, 10),    # 160 tiles: one range per tile, 256 rows per tile
     ("bf16", 4, 2, 128, 256, 5, 64, 1, 0, 1),       # 320 rows: two row chunks
 ]
