@@ -151,3 +151,41 @@ def test_attention_block_of_a_refresh_step_stage_by_stage():
     oy = oracle.linear(wl.to_numpy(out[0, 0]).reshape(M_max, Hq * d), wl.to_numpy(bw.w_o[0]),
                        wl.to_numpy(bw.residual[0, 0]))
     util.compare(util.widen_t(y[0, 0]), oy, "bf16", "block output")
+
+
+@pytest.mark.parametrize("name,layers", [("llama_128k", (0, 13, 31)), ("stress_b4", (0, 31))])
+def test_projections_at_full_size_in_the_benchmark_launch(name, layers):
+    """All 32 layers of the LLaMA-3.1-8B block shapes in one layer-batched launch each (the configuration the
+    benchmark times: 2.7 GB of weights, one input range per tile; batch 4 x 64 rows = one 256-row tile for the
+    stress shape).  Checked on sampled layers: every output of every row against the oracle."""
+    c = wl.CONFIGS[name]
+    L, Hq, Hkv, d, M, batch = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["M"], len(c["ctx"])
+    bw = wl.make_block_weights(name, device="cuda")
+    hid = bw.hidden
+    cfg = make_cfg("bf16", Hq, Hkv, d, L)
+    rng = np.random.default_rng(c["index"])
+    parents = [wl.make_tree(M, c["depth"], c["branch"], rng) for _ in range(batch)]
+    _, _, cos_sin, pos = step_tables(cfg, parents, 0, [M] * batch, list(c["ctx"]), M, d, bw.rope_theta)
+    ws = B.new_workspace(cfg, L, batch, 4096, M)
+    dt = torch.bfloat16
+    q = torch.full((L, batch, M, Hq, d), float("nan"), dtype=dt, device="cuda")
+    k_new = torch.full((L, batch, M, Hkv, d), float("nan"), dtype=dt, device="cuda")
+    v_new = torch.full_like(k_new, float("nan"))
+    y = torch.full((L, batch, M, hid), float("nan"), dtype=dt, device="cuda")
+    attn = bw.x  # any bfloat16 tensor of the right size serves as the attention output here (Hq d = hidden)
+    assert Hq * d == hid
+    B.specpv_qkv_rope(cfg, 0, L, bw.x, hid, bw.w_qkv, cos_sin, batch, M, q, k_new, v_new, ws)
+    B.specpv_o_proj(cfg, 0, L, attn, bw.w_o, hid, bw.residual, batch, M, y, ws)
+    util.sync_status(ws)
+    assert not torch.isnan(q.float()).any() and not torch.isnan(k_new.float()).any()
+    assert not torch.isnan(v_new.float()).any() and not torch.isnan(y.float()).any()
+    for l in layers:
+        wq, wo = wl.to_numpy(bw.w_qkv[l]), wl.to_numpy(bw.w_o[l])
+        for b in range(batch):
+            xb = wl.to_numpy(bw.x[l, b])
+            oq, ok, ov = oracle.qkv_rope(xb, wq, Hq, Hkv, d, pos[b], bw.rope_theta)
+            util.compare(util.widen_t(q[l, b]), oq, "bf16", f"q layer {l} seq {b}")
+            util.compare(util.widen_t(k_new[l, b]), ok, "bf16", f"k layer {l} seq {b}")
+            util.compare(util.widen_t(v_new[l, b]), ov, "bf16", f"v layer {l} seq {b}")
+            util.compare(util.widen_t(y[l, b]), oracle.linear(xb, wo, wl.to_numpy(bw.residual[l, b])), "bf16",
+                         f"block output layer {l} seq {b}")
