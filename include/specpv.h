@@ -285,6 +285,45 @@ specpv_status specpv_o_proj(const specpv_config *cfg, int layer0, int n_layers, 
                             const void *w_o, int hidden, const void *residual, int batch, int M_max, void *y,
                             void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- Full KV cache in host memory ---------------------------------------------------------------
+ * Section 3.3, last paragraph: when device memory is short only the FULL cache is offloaded to host
+ * memory (the partial cache stays resident); a full verification keeps one layer's keys and values
+ * on the device at a time and prefetches the next layer.
+ *
+ * k_host / v_host are page-locked host memory that the device can address (cudaHostAlloc or
+ * cudaHostRegister with the mapped flag; under unified addressing the same pointer serves both
+ * sides), laid out like a K/V pool.  k_stage / v_stage are two layer slots of device memory.
+ * Every other call of this header that takes a specpv_paged_kv also accepts such host pointers as
+ * k_pool / v_pool and then reads or writes the cache over the bus in place: that is how
+ * specpv_commit_accepted appends the accepted rows to an offloaded cache and how
+ * specpv_refresh_partial fetches only the selected blocks (a few percent of the cache) instead of
+ * whole layers.  The summaries (Eq. 1) stay device-resident. */
+typedef struct {
+    const void *k_host;         /* host (device-addressable), [n_layers][n_pages][Hkv][bs][d] */
+    const void *v_host;
+    void *k_stage;              /* device, [2][n_pages][Hkv][bs][d] */
+    void *v_stage;
+    const int32_t *block_table; /* device, [batch][max_blocks] */
+    const int32_t *seq_lens;    /* device, [batch] */
+    int32_t batch;
+    int32_t max_blocks;
+    int32_t n_pages;
+    int32_t max_seq_len;
+} specpv_offloaded_kv;
+
+/* specpv_verify_full over an offloaded cache: for each layer of [layer0, layer0 + n_layers) the layer's
+ * K and V pools are copied host -> device into one of the two slots on `copy_stream` while the attention
+ * of the previous layer runs from the other slot on `stream`.  On return everything is ordered on
+ * `stream` (later work on `stream` sees out / lse; the slots may be reused by a later call on it).
+ * copy_stream must not be a stream that waits on `stream`'s later work; pass a stream of its own
+ * (the same stream is accepted and runs the copies and the attention one after the other).  The call
+ * creates and destroys four CUDA events; it allocates no device memory. */
+specpv_status specpv_verify_full_offloaded(const specpv_config *cfg, int layer0, int n_layers, const void *q,
+                                           const void *k_new, const void *v_new, const uint64_t *tree_mask,
+                                           const int32_t *q_lens, int M_max, const specpv_offloaded_kv *full,
+                                           void *out, float *lse, void *workspace, size_t workspace_bytes,
+                                           void *stream, void *copy_stream);
+
 #ifdef __cplusplus
 }
 #endif

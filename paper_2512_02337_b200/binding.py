@@ -27,7 +27,7 @@ EXPORTS = [
     "specpv_select_mode", "specpv_update_block_summaries", "specpv_score_blocks",
     "specpv_select_partial_kv", "specpv_refresh_partial", "specpv_verify_partial",
     "specpv_verify_full", "specpv_verify_host", "specpv_commit_accepted", "specpv_verify_partial_static",
-    "specpv_rope_table", "specpv_qkv_rope", "specpv_o_proj",
+    "specpv_rope_table", "specpv_qkv_rope", "specpv_o_proj", "specpv_verify_full_offloaded",
 ]
 
 
@@ -268,3 +268,44 @@ def specpv_o_proj(cfg, layer0, n_layers, attn, w_o, hidden, residual, batch, M_m
     _check(lib().specpv_o_proj(ctypes.byref(cfg), layer0, n_layers, _ptr(attn), _ptr(w_o), hidden, _ptr(residual),
                                batch, M_max, _ptr(y), _ptr(workspace), c_size_t(workspace.numel()), _stream(stream)),
            "specpv_o_proj")
+
+
+# ---- full KV cache in host memory -------------------------------------------------------------------------------
+class OffloadedKV(ctypes.Structure):
+    """Mirror of ``specpv_offloaded_kv``."""
+    _fields_ = [("k_host", c_void_p), ("v_host", c_void_p), ("k_stage", c_void_p), ("v_stage", c_void_p),
+                ("block_table", c_void_p), ("seq_lens", c_void_p), ("batch", c_int32), ("max_blocks", c_int32),
+                ("n_pages", c_int32), ("max_seq_len", c_int32)]
+
+
+@dataclass
+class OffloadedCache:
+    """A full cache in pinned host memory plus the two device layer slots a full verification stages through."""
+    k_host: torch.Tensor       # pinned host, [n_layers][n_pages][Hkv][bs][d]
+    v_host: torch.Tensor
+    k_stage: torch.Tensor      # device, [2][n_pages][Hkv][bs][d]
+    v_stage: torch.Tensor
+    block_table: torch.Tensor  # device
+    seq_lens: torch.Tensor     # device
+    max_seq_len: int
+
+    def desc(self) -> OffloadedKV:
+        assert self.k_host.is_pinned() and self.v_host.is_pinned(), "the offloaded pools must be page-locked"
+        batch, max_blocks = self.block_table.shape
+        return OffloadedKV(self.k_host.data_ptr(), self.v_host.data_ptr(), self.k_stage.data_ptr(),
+                           self.v_stage.data_ptr(), self.block_table.data_ptr(), self.seq_lens.data_ptr(), batch,
+                           max_blocks, self.k_host.shape[1], int(self.max_seq_len))
+
+    def as_cache(self) -> Cache:
+        """The host pools as an ordinary cache descriptor (commit and gather address them in place)."""
+        return Cache(self.k_host, self.v_host, self.block_table, self.seq_lens, self.max_seq_len)
+
+
+def specpv_verify_full_offloaded(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max,
+                                 full: OffloadedCache, out, lse, workspace, stream=None, copy_stream=None):
+    d = full.desc()
+    _check(lib().specpv_verify_full_offloaded(ctypes.byref(cfg), layer0, n_layers, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                              _ptr(tree_mask), _ptr(q_lens), M_max, ctypes.byref(d), _ptr(out),
+                                              _ptr(lse), _ptr(workspace), c_size_t(workspace.numel()),
+                                              _stream(stream), _stream(copy_stream)),
+           "specpv_verify_full_offloaded")
