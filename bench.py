@@ -391,6 +391,63 @@ def attention_block(st, peaks, iters=10):
     return res
 
 
+def offloaded_refresh(st, layers=4, iters=3):
+    """The memory-constrained variant (Section 3.3, last paragraph) on the first `layers` layers of the workload: the
+    full cache in page-locked host memory, full verification staged through two device layer slots with the next
+    layer's copy in flight, and the gather of the selected blocks straight from host memory.  Both are bound by the
+    host link, so each is reported with the GB/s it moved over it."""
+    B, w, cfg, M, batch = st["B"], st["w"], st["cfg"], st["M"], st["batch"]
+    c = w.cfg
+    L = min(layers, st["L"])
+    Hkv, d, bs = c["Hkv"], c["d"], c["bs"]
+    dev = w.device
+    dt = wl.torch_dtype(c["dtype"])
+    k_host = torch.empty((L,) + tuple(w.k_pool.shape[1:]), dtype=dt).pin_memory()
+    v_host = torch.empty_like(k_host).pin_memory()
+    k_host.copy_(w.k_pool[:L])
+    v_host.copy_(w.v_pool[:L])
+    stage_shape = (2,) + tuple(w.k_pool.shape[1:])
+    off = B.OffloadedCache(k_host, v_host, torch.zeros(stage_shape, dtype=dt, device=dev),
+                           torch.zeros(stage_shape, dtype=dt, device=dev), w.block_table, w.seq_lens, st["full"].max_seq_len)
+    cfg_l = B.make_config(L, c["Hq"], Hkv, d, bs, c["dtype"], cfg.sink_blocks, cfg.local_blocks, cfg.budget_blocks,
+                          cfg.buffer_tokens)
+    copy_stream = torch.cuda.Stream(device=dev)
+
+    def timed(call):
+        call()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        torch.cuda.synchronize(dev)
+        for a, b in ev:
+            a.record()
+            call()
+            b.record()
+        torch.cuda.synchronize(dev)
+        return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+    layer_bytes = 2 * k_host[0].numel() * k_host.element_size()
+    us_v = timed(lambda: B.specpv_verify_full_offloaded(cfg_l, 0, L, w.q[:L], w.k_new[:L], w.v_new[:L], st["mask"], None, M,
+                                                        off, st["out"][:L], st["lse"][:L], st["ws"],
+                                                        copy_stream=copy_stream))
+    # selection for these layers with this budget into buffers of its own (the step's state is left alone)
+    idx = torch.zeros((L, batch, Hkv, cfg.budget_blocks), dtype=torch.int32, device=dev)
+    count = torch.zeros(batch, dtype=torch.int32, device=dev)
+    plens = torch.zeros(batch, dtype=torch.int32, device=dev)
+    ppb = cfg.budget_blocks + (cfg.buffer_tokens + bs - 1) // bs + 1
+    pk = torch.zeros((L, batch * ppb, Hkv, bs, d), dtype=dt, device=dev)
+    ptable = torch.arange(batch * ppb, dtype=torch.int32, device=dev).reshape(batch, ppb).contiguous()
+    partial = B.Cache(pk, torch.zeros_like(pk), ptable, plens, cfg.budget_blocks * bs + cfg.buffer_tokens)
+    B.specpv_select_partial_kv(cfg_l, L, st["scores"][:L].contiguous(), w.seq_lens, batch, w.max_blocks, idx, count,
+                               st["ws"])
+    us_g = timed(lambda: B.specpv_refresh_partial(cfg_l, off.as_cache(), idx, count, partial, plens, st["ws"]))
+    gathered = L * int(plens.sum()) * Hkv * 2 * d * k_host.element_size()
+    res = {"layers": L,
+           "full_verify_staged": {"us_per_layer": us_v / L, "h2d_gbs": L * layer_bytes / (us_v * 1e-6) / 1e9,
+                                  "bytes_per_layer": layer_bytes},
+           "gather_from_host": {"us_per_layer": us_g / L, "host_read_gbs": gathered / (us_g * 1e-6) / 1e9,
+                                "bytes_per_layer": gathered // L}}
+    del off, k_host, v_host, partial, pk
+    return res
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -451,6 +508,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="skip the per-layer CUDA-graph measurement")
     ap.add_argument("--no-block", action="store_true",
                     help="skip the QKV / output projection measurement (the linear maps either side of the attention)")
+    ap.add_argument("--no-offload", action="store_true",
+                    help="skip the host-offloaded full cache measurement (4 layers staged over the host link)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens)")
     args = ap.parse_args()
 
@@ -502,6 +561,9 @@ def main():
     block = None
     if not args.no_block and rank == 0 and c["dtype"] == "bf16":
         block = attention_block(st, load_peaks())
+    offload = None
+    if not args.no_offload and rank == 0 and c["dtype"] == "bf16":
+        offload = offloaded_refresh(st)
     if rank != 0:
         return 0
 
@@ -550,6 +612,8 @@ def main():
         out["per_layer_cuda_graph"] = graph_times
     if block is not None:
         out["attention_block"] = block
+    if offload is not None:
+        out["offloaded_full_cache"] = offload
     if not args.no_cpu_baseline and world == 1:
         us, sample, cores = oracle_sample(st)
         out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}
