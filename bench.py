@@ -107,10 +107,14 @@ class ClockSampler:
                 "power_w": statistics.median(power) if power else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def build_state(name: str, device, n_layers=None, budget_blocks=None):
+def build_state(name: str, device, n_layers=None, budget_blocks=None, block_tokens=None):
     """Allocate every buffer of the step once (torch owns device memory; nothing is allocated per step)."""
     from paper_2512_02337_b200 import binding as B
     over = {}
+    if block_tokens is not None:  # another page size, the budget kept at the same number of tokens
+        base = wl.CONFIGS[name]
+        over["bs"] = block_tokens
+        over["budget_blocks"] = base["budget_blocks"] * base["bs"] // block_tokens
     if budget_blocks is not None:
         over["budget_blocks"] = budget_blocks
     w = wl.make_workload(name, device=device, n_layers=n_layers, spare_tokens=64, **over)
@@ -503,6 +507,8 @@ def main():
     ap.add_argument("--workload", default="llama_128k", choices=list(wl.CONFIGS))
     ap.add_argument("--layers", type=int, default=None, help="truncate the layer count (profiling only)")
     ap.add_argument("--budget-blocks", type=int, default=None)
+    ap.add_argument("--block-tokens", type=int, default=None, choices=[16, 32, 64],
+                    help="tokens per page (default: the workload's 64; the paper's own block size is 16)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the per-layer CUDA-graph measurement")
@@ -538,7 +544,7 @@ def main():
     else:
         barrier = lambda: None  # noqa: E731
 
-    st = build_state(args.workload, dev, args.layers, args.budget_blocks)
+    st = build_state(args.workload, dev, args.layers, args.budget_blocks, args.block_tokens)
     c = st["w"].cfg
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
     sampler.start()
@@ -553,7 +559,7 @@ def main():
         if not args.no_e2e:
             e2e_ms = e2e_max
     sweep = None
-    if not args.no_sweep and rank == 0 and args.budget_blocks is None and c["dtype"] == "bf16":
+    if not args.no_sweep and rank == 0 and args.budget_blocks is None and args.block_tokens is None and c["dtype"] == "bf16":
         sweep = partial_budget_sweep(st, load_peaks())
     graph_times = None
     if not args.no_graph and rank == 0 and c["dtype"] == "bf16":

@@ -1,4 +1,4 @@
-// Tensor-core verification attention for B200 (sm_100a): bfloat16, head_dim 128, 64-token pages.
+// Tensor-core verification attention for B200 (sm_100a): bfloat16, head_dim 128, pages of 16, 32 or 64 tokens.
 // Tree-masked GQA attention of the step's tokens over a paged cache (paper Section 3.2-3.3,
 // Algorithm 1 "TreeDecode"), used for both the partial and the full cache.
 //
@@ -23,9 +23,8 @@ namespace specpv {
 namespace {
 
 constexpr int kThreadsTc = 384;          // 12 warps
-constexpr int kTileTokens = 128;         // KV tokens per tile (two 64-token pages)
+constexpr int kTileTokens = 128;         // KV tokens per tile (128 / page size pages)
 constexpr int kD = 128;
-constexpr int kPage = 64;
 constexpr int kSlotBytes = 32768;        // one K or V tile: [2 d-halves][128 tokens][64 d] bf16
 constexpr int kStages = 5;
 constexpr int kQBytes = 2 * 32768;       // two row tiles
@@ -39,7 +38,7 @@ struct TcParams {
     CUtensorMap tm_q;      // (d, Hq, tokens)          box (64, G, 128/G)
     CUtensorMap tm_knew;   // (d, Hkv, tokens)         box (64, 1, 64)
     CUtensorMap tm_vnew;
-    CUtensorMap tm_kpool;  // (d, rows)                box (64, 64)
+    CUtensorMap tm_kpool;  // (d, rows)                box (64, page size)
     CUtensorMap tm_vpool;
     const uint64_t* tree_mask;
     const int32_t* q_lens;
@@ -52,6 +51,7 @@ struct TcParams {
     void* workspace;
     int layer0, batch, M_max, mask_words, Hq, Hkv, G, max_blocks, n_pages;
     int n_splits, n_row_groups, R_pad, out_f32;
+    int bs;          // tokens per page (16, 32 or 64)
     uint32_t pool_rows;  // rows of the pool tensor map (an out-of-range row coordinate reads zeros)
     float scale_log2;
 };
@@ -211,44 +211,42 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         __syncwarp();
         const int32_t* table = p.block_table + (size_t)b * p.max_blocks;
         const long long layer_row0 = (long long)(p.layer0 + l) * p.n_pages;
-        // pool row coordinate of a context tile's two pages; the table is read one tile ahead so that
-        // its latency hides behind the wait for a free slot
-        auto page_rows = [&](int j, int* row) {
-            for (int pg = 0; pg < 2; ++pg) {
-                const int blk = (tile_begin + j) * 2 + pg;
-                row[pg] = (int)p.pool_rows;  // out of range: the copy engine fills zeros
-                if (j < n_ctx_tiles && (long long)blk * kPage < seq_len && blk < p.max_blocks) {
-                    const int page = table[blk];
-                    if (page < 0 || page >= p.n_pages) {
-                        if (lane == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
-                    } else {
-                        row[pg] = (int)(((layer_row0 + page) * p.Hkv + h) * kPage);
-                    }
+        bool ok = true;
+        // Pool row coordinate of a context tile's pages (128 / page size of them).  Lane 2 pg + half looks page pg
+        // up and later issues the copy of that page's 64-channel half, so that a tile's copies leave in one pass of
+        // the warp; the table is read one tile ahead so that its latency hides behind the wait for a free slot.
+        const int ppt = kTileTokens / p.bs;
+        const int my_pg = lane >> 1, my_half = lane & 1;
+        auto page_row = [&](int j) {
+            int row = (int)p.pool_rows;  // out of range: the copy engine fills zeros
+            const int blk = (tile_begin + j) * ppt + my_pg;
+            if (my_pg < ppt && j < n_ctx_tiles && (long long)blk * p.bs < seq_len && blk < p.max_blocks) {
+                const int page = table[blk];
+                if (page < 0 || page >= p.n_pages) {
+                    if (my_half == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, b, blk, page, l);
+                } else {
+                    row = (int)(((layer_row0 + page) * p.Hkv + h) * p.bs);
                 }
             }
+            return row;
         };
-        int row_next[2];
-        page_rows(0, row_next);
-        bool ok = true;
+        int row_next = page_row(0);
         uint32_t slot = 0, par = 1;  // ring position of the next use; parity of the release that frees its slot
         for (int j = 0; j < n_tiles; ++j) {
             const bool is_new = j >= n_ctx_tiles;
-            const int row[2] = {row_next[0], row_next[1]};
-            page_rows(j + 1, row_next);
+            const int row_mine = row_next;
+            row_next = page_row(j + 1);
             for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
                 const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
                 if (2 * j + kv >= kStages) ok &= mbar_wait(empty, par, abort_flag, p.workspace, 1);
-                if (lane == 0) {
-                    mbar_expect_tx(full, kSlotBytes);
-                    const uint32_t dst = kv_smem + slot * kSlotBytes;
-                    for (int pg = 0; pg < 2; ++pg)
-                        for (int half = 0; half < 2; ++half) {
-                            const uint32_t d = dst + half * 16384 + pg * 8192;
-                            if (is_new)
-                                tma_load_3d(d, kv ? &p.tm_vnew : &p.tm_knew, half * 64, h, lb * p.M_max + pg * 64, full);
-                            else
-                                tma_load_2d(d, kv ? &p.tm_vpool : &p.tm_kpool, half * 64, row[pg], full);
-                        }
+                const uint32_t dst = kv_smem + slot * kSlotBytes + my_half * 16384;
+                if (lane == 0) mbar_expect_tx(full, kSlotBytes);
+                if (is_new) {  // the step's own tokens: two boxes of 64 rows per half
+                    if (lane < 4)
+                        tma_load_3d(dst + my_pg * 8192, kv ? &p.tm_vnew : &p.tm_knew, my_half * 64, h, lb * p.M_max + my_pg * 64,
+                                    full);
+                } else if (my_pg < ppt) {
+                    tma_load_2d(dst + my_pg * p.bs * 128, kv ? &p.tm_vpool : &p.tm_kpool, my_half * 64, row_mine, full);
                 }
                 __syncwarp();
                 if (++slot == kStages) { slot = 0; par ^= 1; }
@@ -604,11 +602,11 @@ __global__ void __launch_bounds__(32 * kMergeRows) merge_tc_kernel(TcParams p) {
 }  // namespace
 
 bool attention_tc_supported(const AttnArgs& a) {
-    if (a.g.dtype != SPECPV_DTYPE_BF16 || a.g.d != 128 || a.g.bs != 64) return false;
+    if (a.g.dtype != SPECPV_DTYPE_BF16 || a.g.d != 128 || (a.g.bs != 64 && a.g.bs != 32 && a.g.bs != 16)) return false;
     if (a.g.G > 128 || (128 % a.g.G) != 0) return false;
     if (a.M_max > kMaxQTokens) return false;
     // row coordinates of the pool tensor map must fit in a positive int32
-    const unsigned long long rows = (unsigned long long)a.g.n_layers * a.n_pages * a.g.Hkv * 64ull;
+    const unsigned long long rows = (unsigned long long)a.g.n_layers * a.n_pages * a.g.Hkv * (unsigned long long)a.g.bs;
     if (rows >= 0x7FFFFF00ull) return false;
     return get_encode_fn() != nullptr;
 }
@@ -636,11 +634,11 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
         if (!encode_map(&p.tm_knew, a.k_new, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
         if (!encode_map(&p.tm_vnew, a.v_new, 3, dims, strides, box)) return SPECPV_ERR_CUDA;
     }
-    const uint64_t pool_rows = (uint64_t)a.g.n_layers * a.n_pages * Hkv * 64ull;
+    const uint64_t pool_rows = (uint64_t)a.g.n_layers * a.n_pages * Hkv * (uint64_t)a.g.bs;
     {
         uint64_t dims[2] = {128, pool_rows};
         uint64_t strides[1] = {256};
-        uint32_t box[2] = {64, 64};
+        uint32_t box[2] = {64, (uint32_t)a.g.bs};
         if (!encode_map(&p.tm_kpool, a.k_pool, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
         if (!encode_map(&p.tm_vpool, a.v_pool, 2, dims, strides, box)) return SPECPV_ERR_CUDA;
     }
@@ -649,6 +647,7 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
     p.layer0 = a.layer0; p.batch = a.batch; p.M_max = a.M_max; p.mask_words = a.mask_words;
     p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.max_blocks = a.max_blocks; p.n_pages = a.n_pages;
     p.out_f32 = a.g.out_f32;
+    p.bs = a.g.bs;
     p.pool_rows = (uint32_t)pool_rows;
     p.scale_log2 = a.g.scale * kLog2e;
 

@@ -80,6 +80,15 @@ def test_shapes_ragged_context(dtype, Hq, Hkv, d, bs):
     run_case(dtype, Hq, Hkv, d, bs, ctx=[bs * 9 + 5, bs * 4], Ms=[13, 7], seed=Hq + d + bs)
 
 
+@pytest.mark.parametrize("bs", [16, 32])
+def test_small_pages_on_the_tensor_core_path(bs):
+    """16- and 32-token pages (the paper's block size is 16): eight or four pages per 128-token tile, shuffled
+    table, a context long enough to be split over many CTAs with a ragged last page, two layers, refresh rows."""
+    run_case("bf16", 32, 8, 128, bs, ctx=[bs * 531 + bs - 3, bs * 7 + 1, 0], Ms=[60, 9, 2], depth=6, branch=4,
+             n_layers=2, seed=40 + bs)
+    run_case("bf16", 8, 2, 128, bs, ctx=[128 * 20 + 5], Ms=[48], depth=5, branch=4, n_chain=20, seed=41 + bs)
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_empty_context_and_single_node_tree(dtype):
     run_case(dtype, 8, 2, 128, 64, ctx=[0, 1, 64], Ms=[5, 1, 1], seed=3)
