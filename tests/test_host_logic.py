@@ -80,6 +80,51 @@ def test_config_validation_happens_on_the_host():
     assert B.specpv_status_string(0) == "ok" and "capacity" in B.specpv_status_string(4)
 
 
+def test_projection_and_offload_calls_validate_on_the_host():
+    """Bad shapes and null pointers of the linear maps and of the offloaded verification are refused before any CUDA
+    call (so this runs without a GPU); 16-byte aligned host buffers stand in for device pointers."""
+    cfg = B.make_config(n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, block_tokens=64, dtype="fp32", sink_blocks=1,
+                        local_blocks=2, budget_blocks=8, buffer_tokens=64)
+    lib = B.lib()
+    buf = np.zeros(4096, dtype=np.float32)
+    ptr = ctypes.c_void_p(buf.ctypes.data + (-buf.ctypes.data) % 16)
+    size = ctypes.c_size_t(1024)
+
+    def qkv(hidden=512, layer0=0, n_layers=1, x=ptr, cos_sin=ptr, ws=ptr):
+        return lib.specpv_qkv_rope(ctypes.byref(cfg), layer0, n_layers, x, hidden, ptr, cos_sin, 1, 16, ptr, ptr, ptr, ws,
+                                   size, None)
+    assert qkv(hidden=100) == 2          # hidden not a multiple of 16
+    assert qkv(hidden=0) == 2
+    assert qkv(x=None) == 1
+    assert qkv(cos_sin=None) == 1
+    assert qkv(ws=None) == 1
+    assert qkv(layer0=2) == 1            # outside the two layers of the pool
+    assert qkv(n_layers=3) == 1
+    assert qkv(x=ctypes.c_void_p(ptr.value + 4)) == 1  # misaligned
+
+    def o_proj(hidden=512, attn=ptr, y=ptr):
+        return lib.specpv_o_proj(ctypes.byref(cfg), 0, 1, attn, ptr, hidden, None, 1, 16, y, ptr, size, None)
+    assert o_proj(hidden=24) == 2
+    assert o_proj(attn=None) == 1 and o_proj(y=None) == 1
+
+    def table(theta=1.0e4, batch=1, M=16, mask=ptr):
+        return lib.specpv_rope_table(ctypes.byref(cfg), mask, None, ptr, batch, M, ctypes.c_double(theta), ptr, None)
+    assert table(theta=1.0) == 1 and table(theta=float("inf")) == 1 and table(theta=float("nan")) == 1
+    assert table(batch=0) == 1 and table(mask=None) == 1
+    assert table(M=129) == 4             # more rows than the mask words the kernels handle
+
+    off = B.OffloadedKV(ptr, ptr, ptr, ptr, ptr, ptr, 1, 4, 4, 256)
+    def staged(kv=off, q=ptr, layer0=0, n_layers=1, M=16):
+        return lib.specpv_verify_full_offloaded(ctypes.byref(cfg), layer0, n_layers, q, ptr, ptr, ptr, None, M,
+                                                ctypes.byref(kv) if kv is not None else None, ptr, None, ptr, size, None,
+                                                None)
+    assert staged(kv=None) == 1 and staged(q=None) == 1 and staged(n_layers=3) == 1
+    assert staged(kv=B.OffloadedKV(None, ptr, ptr, ptr, ptr, ptr, 1, 4, 4, 256)) == 1
+    assert staged(kv=B.OffloadedKV(ptr, ptr, ptr, ptr, ptr, ptr, 1, 4, 4, 257)) == 4   # longer than the table covers
+    assert staged(M=129) == 4
+    assert staged() == 4                 # a 1 KB workspace cannot hold the split partials
+
+
 def test_workspace_grows_with_the_request():
     cfg = B.make_config(32, 32, 8, 128, 64, "bf16", 1, 2, 64, 80)
     a = B.specpv_workspace_bytes(cfg, 1, 1, 131072, 60)
