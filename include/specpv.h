@@ -224,7 +224,10 @@ specpv_status specpv_verify_partial_static(const specpv_config *cfg, int layer0,
 /* The same step with HOST step tensors (q, k_new, v_new, tree_mask, out, lse are host pointers,
  * ideally pinned): copies the inputs to staging space inside the workspace, runs the attention
  * (mode = SPECPV_MODE_PARTIAL or SPECPV_MODE_FULL selects only validation), copies out/lse back and
- * synchronises the stream before returning.  The KV cache stays device-resident state. */
+ * synchronises the stream before returning.  The KV cache stays device-resident state.  The layers go
+ * through in up to eight groups so that one group's attention overlaps the next group's input copy and
+ * the previous group's output copy; the two copy streams this needs are created on the first call on
+ * each device and kept until the process exits. */
 specpv_status specpv_verify_host(const specpv_config *cfg, int mode, int layer0, int n_layers,
                                  const void *q_host, const void *k_new_host, const void *v_new_host,
                                  const uint64_t *tree_mask_host, int M_max, const specpv_paged_kv *kv,

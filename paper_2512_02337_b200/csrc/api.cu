@@ -127,6 +127,25 @@ static specpv_status verify_common(const specpv_config* cfg, int layer0, int n_l
     return launch_attention_simt(a, s);
 }
 
+// Two copy streams per device for specpv_verify_host, created on first use and kept for the life of the process.
+struct HostCopyStreams {
+    cudaStream_t in, out;
+};
+static HostCopyStreams* host_copy_streams() {
+    static std::mutex mu;
+    static HostCopyStreams per_device[64];
+    static bool made[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!made[dev]) {
+        if (cudaStreamCreateWithFlags(&per_device[dev].in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&per_device[dev].out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        made[dev] = true;
+    }
+    return &per_device[dev];
+}
+
 }  // namespace specpv
 
 using namespace specpv;
@@ -399,24 +418,68 @@ SPECPV_EXPORT specpv_status specpv_verify_host(const specpv_config* cfg, int mod
     StagingPlan sp = plan_staging(g, n_layers, kv->batch, M_max);
     char* stage = reinterpret_cast<char*>(workspace) + w.staging_off;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const size_t rows = (size_t)n_layers * kv->batch * M_max;
-    const size_t q_bytes = rows * g.Hq * g.d * g.es, kv_bytes = rows * g.Hkv * g.d * g.es;
+    const size_t rows_l = (size_t)kv->batch * M_max;  // rows of one layer
+    const size_t q_l = rows_l * g.Hq * g.d * g.es, kv_l = rows_l * g.Hkv * g.d * g.es;
+    const size_t out_l = rows_l * g.Hq * g.d * g.out_es, lse_l = rows_l * g.Hq * sizeof(float);
     const size_t mask_bytes = (size_t)kv->batch * M_max * ((M_max + 63) / 64) * sizeof(uint64_t);
-    if (cudaMemcpyAsync(stage + sp.q, q_host, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SPECPV_ERR_CUDA;
-    if (cudaMemcpyAsync(stage + sp.k_new, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SPECPV_ERR_CUDA;
-    if (cudaMemcpyAsync(stage + sp.v_new, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SPECPV_ERR_CUDA;
-    if (cudaMemcpyAsync(stage + sp.mask, tree_mask_host, mask_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SPECPV_ERR_CUDA;
-    st = verify_common(cfg, layer0, n_layers, stage + sp.q, stage + sp.k_new, stage + sp.v_new,
-                       reinterpret_cast<const uint64_t*>(stage + sp.mask), nullptr, M_max, kv, stage + sp.out,
-                       lse_host ? reinterpret_cast<float*>(stage + sp.lse) : nullptr, workspace,
-                       w.partial_off + w.partial_bytes, stream, mode == SPECPV_MODE_PARTIAL);
+
+    // The layers go through in groups: while one group's attention runs on `stream`, the next group's inputs arrive
+    // on a copy-in stream and the previous group's outputs leave on a copy-out stream (the host link carries both
+    // directions at once).  The two copy streams are created once per device and kept.
+    HostCopyStreams* cs = host_copy_streams();
+    if (!cs) return SPECPV_ERR_CUDA;
+    constexpr int kMaxGroups = 8;
+    const int n_groups = n_layers < kMaxGroups ? n_layers : kMaxGroups;
+    const int per_group = (n_layers + n_groups - 1) / n_groups;
+    cudaEvent_t begin = nullptr, in_done[kMaxGroups] = {}, run_done[kMaxGroups] = {}, out_done = nullptr;
+    bool ok = cudaEventCreateWithFlags(&begin, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&out_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < n_groups && ok; ++i)
+        ok = cudaEventCreateWithFlags(&in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&run_done[i], cudaEventDisableTiming) == cudaSuccess;
+    // the staging area may still be in use by earlier work on `stream`
+    ok = ok && cudaEventRecord(begin, s) == cudaSuccess && cudaStreamWaitEvent(cs->in, begin, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(cs->out, begin, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(stage + sp.mask, tree_mask_host, mask_bytes, cudaMemcpyHostToDevice, cs->in) == cudaSuccess;
+    int n_used = 0;
+    for (int i = 0; i < n_groups && ok && st == SPECPV_OK; ++i) {
+        const int l0 = i * per_group, nl = n_layers - l0 < per_group ? n_layers - l0 : per_group;
+        if (nl <= 0) break;
+        n_used = i + 1;
+        ok = cudaMemcpyAsync(stage + sp.q + l0 * q_l, static_cast<const char*>(q_host) + l0 * q_l, nl * q_l,
+                             cudaMemcpyHostToDevice, cs->in) == cudaSuccess &&
+             cudaMemcpyAsync(stage + sp.k_new + l0 * kv_l, static_cast<const char*>(k_new_host) + l0 * kv_l, nl * kv_l,
+                             cudaMemcpyHostToDevice, cs->in) == cudaSuccess &&
+             cudaMemcpyAsync(stage + sp.v_new + l0 * kv_l, static_cast<const char*>(v_new_host) + l0 * kv_l, nl * kv_l,
+                             cudaMemcpyHostToDevice, cs->in) == cudaSuccess &&
+             cudaEventRecord(in_done[i], cs->in) == cudaSuccess && cudaStreamWaitEvent(s, in_done[i], 0) == cudaSuccess;
+        if (!ok) break;
+        st = verify_common(cfg, layer0 + l0, nl, stage + sp.q + l0 * q_l, stage + sp.k_new + l0 * kv_l,
+                           stage + sp.v_new + l0 * kv_l, reinterpret_cast<const uint64_t*>(stage + sp.mask), nullptr, M_max, kv,
+                           stage + sp.out + l0 * out_l,
+                           lse_host ? reinterpret_cast<float*>(stage + sp.lse + l0 * lse_l) : nullptr, workspace,
+                           w.partial_off + w.partial_bytes, stream, mode == SPECPV_MODE_PARTIAL);
+        if (st != SPECPV_OK) break;
+        ok = cudaEventRecord(run_done[i], s) == cudaSuccess && cudaStreamWaitEvent(cs->out, run_done[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync(static_cast<char*>(out_host) + l0 * out_l, stage + sp.out + l0 * out_l, nl * out_l,
+                             cudaMemcpyDeviceToHost, cs->out) == cudaSuccess;
+        if (ok && lse_host)
+            ok = cudaMemcpyAsync(reinterpret_cast<char*>(lse_host) + l0 * lse_l, stage + sp.lse + l0 * lse_l, nl * lse_l,
+                                 cudaMemcpyDeviceToHost, cs->out) == cudaSuccess;
+    }
+    // everything is joined back onto `stream` before the call returns (also on the error paths: no copy may outlive it)
+    const bool joined = cudaEventRecord(out_done, cs->out) == cudaSuccess && cudaStreamWaitEvent(s, out_done, 0) == cudaSuccess;
+    const bool in_idle = cudaStreamSynchronize(cs->in) == cudaSuccess;
+    const bool synced = cudaStreamSynchronize(s) == cudaSuccess && (joined || cudaStreamSynchronize(cs->out) == cudaSuccess);
+    (void)n_used;
+    if (begin) cudaEventDestroy(begin);
+    if (out_done) cudaEventDestroy(out_done);
+    for (int i = 0; i < kMaxGroups; ++i) {
+        if (in_done[i]) cudaEventDestroy(in_done[i]);
+        if (run_done[i]) cudaEventDestroy(run_done[i]);
+    }
     if (st != SPECPV_OK) return st;
-    if (cudaMemcpyAsync(out_host, stage + sp.out, rows * g.Hq * g.d * g.out_es, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return SPECPV_ERR_CUDA;
-    if (lse_host && cudaMemcpyAsync(lse_host, stage + sp.lse, rows * g.Hq * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return SPECPV_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return SPECPV_ERR_CUDA;
-    return SPECPV_OK;
+    return ok && in_idle && synced ? SPECPV_OK : SPECPV_ERR_CUDA;
 }
 
 SPECPV_EXPORT specpv_status specpv_commit_accepted(const specpv_config* cfg, int layer0, int n_layers,

@@ -211,3 +211,39 @@ def test_selection_alone_on_synthetic_scores_with_ties_and_nan(nb, budget):
             for h in range(Hkv):
                 want = oracle.select(sc[l, b, h, :n].astype(np.float64), 1, 2, budget)
                 assert np.array_equal(got[l, b, h, :len(want)], want), (l, b, h)
+
+
+@pytest.mark.parametrize("name,L,over", [("tiny_fp32", 1, {}), ("llama_32k", 5, dict(ctx=[5000])),
+                                         ("llama_32k", 11, dict(ctx=[1500])), ("stress_b4", 3, dict(ctx=[900, 2100, 64, 1300]))])
+def test_verify_host_matches_the_device_call_and_the_oracle(name, L, over):
+    """The end-to-end entry point (pinned host step tensors in, host outputs back; layers pipelined in groups of
+    1 and 2 with a short last group) against the device-pointer call and, on one layer, the oracle."""
+    w = wl.make_workload(name, device="cuda", n_layers=L, spare_tokens=256, **over)  # the bytes of run_pipeline's caches
+    c = w.cfg
+    Hq, d, M, batch = c["Hq"], c["d"], c["M"], w.batch
+    cfg = util.config_for(w)
+    full = util.full_cache(w)
+    ws = B.new_workspace(cfg, L, batch, int(max(c["ctx"])) + 256, M)
+    mask = util.device_masks(w.parents, M)
+    out_d = torch.zeros((L, batch, M, Hq, d), dtype=torch.float32, device="cuda")
+    lse_d = torch.zeros((L, batch, M, Hq), dtype=torch.float32, device="cuda")
+    B.specpv_verify_full(cfg, 0, L, w.q, w.k_new, w.v_new, mask, None, M, full, out_d, lse_d, ws)
+    host = [t.cpu().pin_memory() for t in (w.q, w.k_new, w.v_new)]
+    mask_h = mask.cpu().pin_memory()
+    out_h = torch.full((L, batch, M, Hq, d), float("nan"), dtype=torch.float32).pin_memory()
+    lse_h = torch.full((L, batch, M, Hq), float("nan"), dtype=torch.float32).pin_memory()
+    for _ in range(2):  # twice: the staging area and the copy streams are reused
+        B.specpv_verify_host(cfg, B.MODE_FULL, 0, L, host[0], host[1], host[2], mask_h, M, full, out_h, lse_h, ws)
+    util.sync_status(ws)
+    # the layer groups may be split over the KV range differently from the one-launch call: two results that are each
+    # within the bar of the oracle, not bit-equal to each other
+    tol = 2e-5 if c["dtype"] == "fp32" else 4e-2
+    assert torch.isfinite(out_h).all() and torch.isfinite(lse_h).all()
+    assert (out_h - out_d.cpu()).abs().max().item() <= tol
+    assert (lse_h - lse_d.cpu()).abs().max().item() <= tol
+    l, b = L - 1, batch - 1
+    o_out, o_lse = oracle.tree_attention(wl.to_numpy(w.q[l, b]), wl.to_numpy(w.k_new[l, b]), wl.to_numpy(w.v_new[l, b]),
+                                         oracle.tree_mask(w.parents[b]), wl.to_numpy(w.k_pool[l]),
+                                         wl.to_numpy(w.v_pool[l]), wl.to_numpy(w.block_table[b]), int(c["ctx"][b]))
+    util.compare(out_h[l, b].numpy(), o_out, c["dtype"], "verify_host")
+    np.testing.assert_allclose(lse_h[l, b].numpy(), o_lse, atol=5e-3)
