@@ -5,8 +5,9 @@
 // One CTA owns one (layer, sequence, KV head, KV split, row group).  All G query heads of the KV
 // head times up to 2*(128/G) step tokens are packed into two 128-row tiles, so QK^T and PV are
 // dense 128x128x128 contractions:
-//   warp 0      TMA producer: Q once, then K and V tiles of 128 tokens (two pages) through the
-//               block table into a ring of 32 KB shared-memory slots (128-byte swizzle)
+//   warp 0      TMA producer: Q once, then K and V tiles of 128 tokens (2, 4 or 8 pages, one copy per page
+//               and 64-channel half, each issued by its own lane) through the block table into a ring of
+//               32 KB shared-memory slots (128-byte swizzle)
 //   warp 1      MMA issuer: tcgen05.mma  S_t = Q_t K^T  (both operands in shared memory) and
 //               O_t += P_t V (P read from tensor memory, V MN-major from shared memory)
 //   warps 4-7   softmax of row tile 0, warps 8-11 of row tile 1: one thread per row reads S from
