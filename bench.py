@@ -586,7 +586,8 @@ def main():
                 "peak": peaks["hbm_gbs"] if bound == "hbm" else peaks["bf16_tflops"],
                 "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
                 "frac": (achieved_gbs / peaks["hbm_gbs"]) if bound == "hbm" else achieved_tf / peaks["bf16_tflops"],
-                "peak_source": peaks["source"], "traffic": ncu_traffic_bytes(args.workload, st["L"]),
+                "peak_source": peaks["source"],
+                "traffic": ncu_traffic_bytes(args.workload, st["L"]) if args.block_tokens in (None, 64) else None,
                 "launch_us": full_avg_s * 1e6, "bound_us": max(t_hbm, t_tensor) * 1e6,
                 "achieved_gbs": achieved_gbs, "achieved_tflops": achieved_tf,
                 "frac_of_bound": max(t_hbm, t_tensor) / full_avg_s}
