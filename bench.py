@@ -452,6 +452,48 @@ def offloaded_refresh(st, layers=4, iters=3):
     return res
 
 
+def score_variants(st, peaks, iters=10):
+    """Block scoring and selection in their variants (Eq. 3's reductions mean / max / last, Eq. 2 as printed and in
+    its channel-wise form, selection per head and shared by the heads), each call alone over all layers.  Scoring
+    reads the summaries once: `frac` is against the HBM time of those bytes."""
+    B, w, L, M, batch = st["B"], st["w"], st["L"], st["M"], st["batch"]
+    c = w.cfg
+    Hq, Hkv, d, bs = c["Hq"], c["Hkv"], c["d"], c["bs"]
+    base = st["cfg"]
+    dev = w.device
+    nbytes = 2 * st["kmax"].numel() * st["kmax"].element_size() * sum((x + bs - 1) // bs for x in c["ctx"]) \
+        // (batch * w.max_blocks)
+
+    def timed(call):
+        for _ in range(3):
+            call()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+        torch.cuda.synchronize(dev)
+        for a, b in ev:
+            a.record()
+            call()
+            b.record()
+        torch.cuda.synchronize(dev)
+        return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+    scores = torch.zeros_like(st["scores"])
+    idx = torch.zeros_like(st["idx"])
+    count = torch.zeros_like(st["count"])
+    res = {}
+    for label, reduce, mode in (("mean", 0, 0), ("max", 1, 0), ("last", 2, 0), ("mean_channelwise", 0, 1)):
+        cfg = B.make_config(L, Hq, Hkv, d, bs, c["dtype"], base.sink_blocks, base.local_blocks, base.budget_blocks,
+                            base.buffer_tokens, reduce=reduce, score_mode=mode)
+        us = timed(lambda: B.specpv_score_blocks(cfg, 0, L, w.q, None, M, st["last_query"], st["kmax"], st["kmin"],
+                                                 st["full"], scores, st["ws"]))
+        res["scores_" + label] = {"us": us, "frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6)}
+    for label, shared in (("per_head", 0), ("shared_heads", 1)):
+        cfg = B.make_config(L, Hq, Hkv, d, bs, c["dtype"], base.sink_blocks, base.local_blocks, base.budget_blocks,
+                            base.buffer_tokens, select_shared=shared)
+        us = timed(lambda: B.specpv_select_partial_kv(cfg, L, st["scores"], w.seq_lens, batch, w.max_blocks, idx, count,
+                                                      st["ws"]))
+        res["select_" + label] = {"us": us}
+    return res
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -516,7 +558,7 @@ def main():
                     help="skip the QKV / output projection measurement (the linear maps either side of the attention)")
     ap.add_argument("--no-offload", action="store_true",
                     help="skip the host-offloaded full cache measurement (4 layers staged over the host link)")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the partial-budget sweep (2048/4096/8192 tokens) and the score / selection variants")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -567,6 +609,9 @@ def main():
     block = None
     if not args.no_block and rank == 0 and c["dtype"] == "bf16":
         block = attention_block(st, load_peaks())
+    variants = None
+    if not args.no_sweep and rank == 0 and c["dtype"] == "bf16":
+        variants = score_variants(st, load_peaks())
     offload = None
     if not args.no_offload and rank == 0 and c["dtype"] == "bf16":
         offload = offloaded_refresh(st)
@@ -621,6 +666,8 @@ def main():
         out["attention_block"] = block
     if offload is not None:
         out["offloaded_full_cache"] = offload
+    if variants is not None:
+        out["score_variants"] = variants
     if not args.no_cpu_baseline and world == 1:
         us, sample, cores = oracle_sample(st)
         out["cpu_baseline"] = {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample}

@@ -261,8 +261,8 @@ SPECPV_EXPORT specpv_status specpv_score_blocks(const specpv_config* cfg, int la
     p.workspace = workspace;
     p.score_mode = g.score_mode;
     const int max_nb = (kv->max_seq_len + g.bs - 1) / g.bs;
-    // the tensor-core kernel computes Eq. 2 as printed; the channel-wise form runs on the SIMT kernel
-    if (g.score_mode == 0 && scores_tc_supported(g.dtype, g.d, g.G, M_max) && aligned16(q) && aligned16(kmax) && aligned16(kmin))
+    // both forms of Eq. 2 run on the tensor-core kernel (the channel-wise one as Kmax . q+ + Kmin . q-)
+    if (scores_tc_supported(g.dtype, g.d, g.G, M_max) && aligned16(q) && aligned16(kmax) && aligned16(kmin))
         return launch_scores_tc(p, n_layers, g.n_layers, max_nb, reinterpret_cast<cudaStream_t>(stream));
     return launch_scores(p, n_layers, max_nb, g.dtype, g.d, reinterpret_cast<cudaStream_t>(stream));
 }

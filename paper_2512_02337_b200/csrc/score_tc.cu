@@ -1,5 +1,9 @@
 // Block scores on the tensor cores (paper Eq. 2-3): s_i = f_r max(q_r . Kmax_i, q_r . Kmin_i) for
-// bfloat16 summaries with head_dim 128.
+// bfloat16 summaries with head_dim 128, and the channel-wise form s_i = f_r sum_c max(q_rc Kmax_ic, q_rc Kmin_ic).
+// Because Kmax >= Kmin in every channel, the channel-wise maximum takes Kmax where q is positive and Kmin where it
+// is negative, so that form is the single contraction  Kmax . q+  +  Kmin . q-  with q+ = max(q, 0), q- = min(q, 0)
+// (both exact in bfloat16): the CTA splits Q by sign in shared memory and accumulates both products into one
+// accumulator.
 //
 // Per (layer, sequence, KV head) the two products are dense contractions
 //     Dmax[128 blocks x R] = Kmax_tile[128 x 128] * Q^T[128 x R],   Dmin likewise with Kmin,
@@ -49,10 +53,13 @@ struct __align__(8) ScoreBarriers {
     uint64_t sum_empty[kScoreStages];
     uint64_t d_full;
     uint64_t d_empty;
+    uint64_t q_split;  // channel-wise form: the epilogue warps have split Q by sign
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// kCw: the channel-wise form (a compile-time switch, so that the printed form's code is exactly what it was).
+template <bool kCw>
 __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __grid_constant__ ScoreTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -78,7 +85,10 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     if (col_end <= col_begin) return;
 
     const uint32_t q_smem = smem_u32(smem);
-    const uint32_t sum_smem = q_smem + kScoreQBytes;
+    // channel-wise form: q- takes the place of the second summary stage, the summaries go through a single stage
+    constexpr int stages = kCw ? 1 : kScoreStages;
+    const uint32_t qneg_smem = q_smem + kScoreQBytes;
+    const uint32_t sum_smem = q_smem + (kCw ? 2 : 1) * kScoreQBytes;
     volatile int* abort_flag = &bars.abort_flag;
 
     if (threadIdx.x == 0) {
@@ -89,6 +99,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         }
         mbar_init(smem_u32(&bars.d_full), 1);
         mbar_init(smem_u32(&bars.d_empty), 4);  // one arrival per epilogue warp
+        mbar_init(smem_u32(&bars.q_split), 4);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -112,7 +123,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         const int n_q_tiles = p.n_cols > 128 ? 2 : 1;
         const int row0 = (((p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks;
         auto load_tile = [&](int i) {  // lane 0 only
-            const int slot = i % kScoreStages;
+            const int slot = i % stages;
             const uint32_t full = smem_u32(&bars.sum_full[slot]);
             mbar_expect_tx(full, 2 * kSumTileBytes);
             const uint32_t dst = sum_smem + slot * 2 * kSumTileBytes;
@@ -136,18 +147,20 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
         const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | (1u << 16);
         const uint32_t sum_lo = ((sum_smem >> 4) & 0x3FFFu) | (1u << 16);
+        const uint32_t qneg_lo = ((qneg_smem >> 4) & 0x3FFFu) | (1u << 16);
         bool ok = mbar_wait(qbar, 0, abort_flag, p.workspace, 20);
+        if (kCw) ok &= mbar_wait(smem_u32(&bars.q_split), 0, abort_flag, p.workspace, 25);
         for (int i = 0; i < n_tiles; ++i) {
-            if (i + 1 < n_tiles) {
+            if (stages > 1 && i + 1 < n_tiles) {  // the next tile goes into the other stage while this one is used
                 const int use = i + 1;
-                if (use >= kScoreStages)
-                    ok &= mbar_wait(smem_u32(&bars.sum_empty[use % kScoreStages]), ((use / kScoreStages) - 1) & 1,
+                if (use >= stages)
+                    ok &= mbar_wait(smem_u32(&bars.sum_empty[use % stages]), ((use / stages) - 1) & 1,
                                     abort_flag, p.workspace, 21);
                 if (lane == 0 && ok) load_tile(use);
                 __syncwarp();
             }
-            const int slot = i % kScoreStages;
-            ok &= mbar_wait(smem_u32(&bars.sum_full[slot]), (i / kScoreStages) & 1, abort_flag, p.workspace, 22);
+            const int slot = i % stages;
+            ok &= mbar_wait(smem_u32(&bars.sum_full[slot]), (i / stages) & 1, abort_flag, p.workspace, 22);
             if (i > 0) ok &= mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
             tc_fence_after();
             if (lane == 0) {
@@ -158,12 +171,24 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                     const uint32_t b_off = (uint32_t)((kk >> 2) * 32768 + (kk & 3) * 32) >> 4;
                     const uint64_t bdesc = ((uint64_t)desc_hi << 32) | (q_lo + b_off);
                     mma_ss(tmem, ((uint64_t)desc_hi << 32) | (a_max + a_off), bdesc, idesc, kk > 0);
-                    mma_ss(tmem + 256, ((uint64_t)desc_hi << 32) | (a_min + a_off), bdesc, idesc, kk > 0);
+                    // channel-wise: Kmin . q- joins Kmax . q+ in the same accumulator
+                    if (kCw)
+                        mma_ss(tmem, ((uint64_t)desc_hi << 32) | (a_min + a_off), ((uint64_t)desc_hi << 32) | (qneg_lo + b_off),
+                               idesc, 1);
+                    else
+                        mma_ss(tmem + 256, ((uint64_t)desc_hi << 32) | (a_min + a_off), bdesc, idesc, kk > 0);
                 }
                 tc_commit(smem_u32(&bars.d_full));
                 tc_commit(smem_u32(&bars.sum_empty[slot]));
             }
             __syncwarp();
+            if (stages == 1 && i + 1 < n_tiles) {
+                // a single stage: the next tile can only follow the contractions just issued (their completion is
+                // release number i of the stage); it still overlaps this tile's reduction
+                ok &= mbar_wait(smem_u32(&bars.sum_empty[0]), i & 1, abort_flag, p.workspace, 21);
+                if (lane == 0 && ok) load_tile(i + 1);
+                __syncwarp();
+            }
         }
         (void)ok;
     } else if (warp >= 2) {
@@ -172,6 +197,29 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         const int blk_in_tile = q * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         bool ok = true;
+        if (kCw) {
+            // split Q by sign in place: q+ stays where Q landed, q- goes to the buffer behind it (same swizzled layout,
+            // the split is element-wise).  A bfloat16 is negative when its top bit is set.
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 26));
+            uint4* qp = reinterpret_cast<uint4*>(smem);
+            uint4* qn = reinterpret_cast<uint4*>(smem + kScoreQBytes);
+            for (int v = threadIdx.x - 64; v < kScoreQBytes / 16; v += 128) {
+                const uint4 w = qp[v];
+                const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+                uint32_t pos[4], neg[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t m = ((in[e] >> 15) & 0x00010001u) * 0xFFFFu;  // all ones in the negative halves
+                    neg[e] = in[e] & m;
+                    pos[e] = in[e] & ~m;
+                }
+                qp[v] = make_uint4(pos[0], pos[1], pos[2], pos[3]);
+                qn[v] = make_uint4(neg[0], neg[1], neg[2], neg[3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor pipe reads these through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.q_split));
+        }
         for (int i = 0; i < n_tiles && ok; ++i) {
             ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full), i & 1, abort_flag, p.workspace, 24));
             if (!ok) break;
@@ -186,9 +234,15 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                 uint32_t vmax[64], vmin[64];
                 TMEM_LD32(tmem + lane_addr + c0, vmax);
                 TMEM_LD32(tmem + lane_addr + c0 + 32, (vmax + 32));
-                TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
-                TMEM_LD32(tmem + lane_addr + 256 + c0 + 32, (vmin + 32));
+                if (!kCw) {
+                    TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
+                    TMEM_LD32(tmem + lane_addr + 256 + c0 + 32, (vmin + 32));
+                }
                 tmem_wait_ld();
+                if (kCw) {  // one accumulator already holds the score: max(x, x) = x below
+#pragma unroll
+                    for (int k = 0; k < 64; ++k) vmin[k] = vmax[k];
+                }
                 const bool whole = c0 >= col_begin && c0 + 64 <= col_end;  // warp-uniform
                 if (whole && !is_max) {
 #pragma unroll
@@ -238,7 +292,8 @@ specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_l
                                cudaStream_t stream) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(scores_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(scores_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess)
             return SPECPV_ERR_CUDA;
         attr_set = true;
     }
@@ -274,7 +329,10 @@ specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_l
     p.tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
     ctas_x = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
     dim3 grid(ctas_x, sp.Hkv, n_layers_call * sp.batch);
-    scores_tc_kernel<<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
+    if (sp.score_mode == 1)
+        scores_tc_kernel<true><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
+    else
+        scores_tc_kernel<false><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
     return SPECPV_OK;

@@ -33,13 +33,13 @@ def check_rows(got_out, got_lse, q, kn, vn, parents, rows, kp, vp, table, seq_le
     np.testing.assert_allclose(got_lse[closed], o_lse, atol=5e-3, err_msg=what)
 
 
-def run_full_size(name, layers, budgets):
+def run_full_size(name, layers, budgets, score_mode=0):
     dev = torch.device("cuda")
     w = wl.make_workload(name, device=dev, spare_tokens=64)
     c = w.cfg
     L, Hq, Hkv, d, bs, M, batch = c["n_layers"], c["Hq"], c["Hkv"], c["d"], c["bs"], c["M"], w.batch
     rng = np.random.default_rng(c["index"])
-    cfg = util.config_for(w)
+    cfg = util.config_for(w, score_mode=score_mode)
     full = util.full_cache(w)
     full.max_seq_len = int(max(c["ctx"])) + 64
     ws = B.new_workspace(cfg, L, batch, full.max_seq_len, M)
@@ -72,14 +72,14 @@ def run_full_size(name, layers, budgets):
             okmax, okmin = oracle.block_summaries(kp, table[b], sl)
             assert np.array_equal(util.widen_t(kmax[l, b])[:, :nb], okmax)
             assert np.array_equal(util.widen_t(kmin[l, b])[:, :nb], okmin)
-            osc = oracle.block_scores(qn[b], okmax, okmin, Hkv, reduce=0, last_query=0)
+            osc = oracle.block_scores(qn[b], okmax, okmin, Hkv, reduce=0, last_query=0, score_mode=score_mode)
             np.testing.assert_allclose(scores_g[l, b, :, :nb], osc, rtol=2e-3, atol=2e-2)
             check_rows(got_out[b], got_lse[b], qn[b], knn[b], vnn[b], w.parents[b], rows[b], kp, vp, table[b], sl,
                        f"{name} full l{l} b{b}")
 
     # selection / gather / partial verification for every budget of the sweep
     for budget in budgets:
-        cfgb = util.config_for(w, budget_blocks=budget)
+        cfgb = util.config_for(w, budget_blocks=budget, score_mode=score_mode)
         idx = torch.full((L, batch, Hkv, budget), -7, dtype=torch.int32, device=dev)
         count = torch.zeros(batch, dtype=torch.int32, device=dev)
         ppb = budget + (cfgb.buffer_tokens + bs - 1) // bs + 1
@@ -121,6 +121,11 @@ def run_full_size(name, layers, budgets):
 
 def test_llama_32k_all_layers_sampled():
     run_full_size("llama_32k", layers=[0, 31], budgets=[64])
+
+
+def test_llama_32k_channelwise_scores_several_tiles_per_cta():
+    # the channel-wise form of Eq. 2 at full size: 256 heads leave two CTAs per head, two 128-block tiles each
+    run_full_size("llama_32k", layers=[3, 31], budgets=[64], score_mode=1)
 
 
 def test_llama_128k_all_layers_sampled_budget_sweep():
