@@ -45,6 +45,8 @@ struct ScoreTcParams {
     float* scores;
     void* workspace;
     int layer0, batch, M_max, Hkv, G, bs, max_blocks, reduce, tiles_per_cta, n_cols;
+    int tok0, tok_n;  // this pass covers step tokens [tok0, tok0 + tok_n): 256 query rows at most (the accumulator's columns)
+    int accumulate;   // a later pass: combine with the scores the earlier passes left
 };
 
 struct __align__(8) ScoreBarriers {
@@ -75,14 +77,19 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     const int n_tiles = tile_end - tile_begin;
     int M = p.q_lens ? p.q_lens[b] : p.M_max;
     M = min(max(M, 0), p.M_max);
-    int col_begin = 0, col_end = M * p.G;  // query rows r = token * G + head, one accumulator column each
+    // query rows r = token * G + head of this pass's tokens, one accumulator column each
+    int col_begin = 0, col_end = min(max(M - p.tok0, 0), p.tok_n) * p.G;
+    int denom = M * p.G;  // rows the mean runs over (all passes together)
     if (p.reduce == SPECPV_REDUCE_LAST) {
         int last = p.last_query ? p.last_query[b] : 0;
         last = min(max(last, 0), max(M - 1, 0));
-        col_begin = last * p.G;
+        if (M <= 0 || last < p.tok0 || last >= p.tok0 + p.tok_n) return;  // another pass holds that row
+        col_begin = (last - p.tok0) * p.G;
         col_end = col_begin + p.G;
+        denom = p.G;
     }
     if (col_end <= col_begin) return;
+    const bool combine = p.accumulate && p.reduce != SPECPV_REDUCE_LAST;
 
     const uint32_t q_smem = smem_u32(smem);
     // channel-wise form: q- takes the place of the second summary stage, the summaries go through a single stage
@@ -138,7 +145,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
             for (int t = 0; t < n_q_tiles; ++t)
                 for (int half = 0; half < 2; ++half)
                     tma_load_3d(q_smem + half * 32768 + t * 16384, &p.tm_q, half * 64, h * p.G,
-                                lb * p.M_max + t * tok_per_tile, qbar);
+                                lb * p.M_max + p.tok0 + t * tok_per_tile, qbar);
             load_tile(0);
         }
         __syncwarp();
@@ -267,8 +274,10 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
             if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty));
             const int blk = (tile_begin + i) * kTileBlocks + blk_in_tile;
             if (blk < nb) {
-                if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)(col_end - col_begin);
-                p.scores[((size_t)lb * p.Hkv + h) * p.max_blocks + blk] = red;
+                float* dst = p.scores + ((size_t)lb * p.Hkv + h) * p.max_blocks + blk;
+                if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)denom;
+                if (combine) red = is_max ? fmaxf(red, *dst) : red + *dst;
+                *dst = red;
             }
         }
     }
@@ -284,7 +293,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
 }  // namespace
 
 bool scores_tc_supported(int dtype, int d, int G, int M_max) {
-    return dtype == SPECPV_DTYPE_BF16 && d == 128 && G <= 128 && (128 % G) == 0 && M_max * G <= 256 &&
+    return dtype == SPECPV_DTYPE_BF16 && d == 128 && G <= 128 && (128 % G) == 0 && M_max * G <= 4 * 256 &&
            tc::get_encode_fn() != nullptr;
 }
 
@@ -318,8 +327,6 @@ specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_l
     p.workspace = sp.workspace;
     p.layer0 = sp.layer0; p.batch = sp.batch; p.M_max = sp.M_max; p.Hkv = sp.Hkv; p.G = sp.G; p.bs = sp.bs;
     p.max_blocks = sp.max_blocks; p.reduce = sp.reduce;
-    const int R = sp.M_max * sp.G;
-    p.n_cols = R <= 128 ? 128 : 256;  // accumulator columns = query rows, padded to whole 128-row Q tiles
     const int n_tiles = (max_nb + kTileBlocks - 1) / kTileBlocks;
     const int heads = sp.Hkv * n_layers_call * sp.batch;
     // enough CTAs to fill the machine, but at least a few tiles each so that Q is amortised
@@ -329,12 +336,21 @@ specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_l
     p.tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
     ctas_x = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
     dim3 grid(ctas_x, sp.Hkv, n_layers_call * sp.batch);
-    if (sp.score_mode == 1)
-        scores_tc_kernel<true><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
-    else
-        scores_tc_kernel<false><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
-    count_launch();
+    // The accumulator holds 256 query rows; a step with more (the chain and the tree of a refresh) goes through in
+    // passes over the step's tokens, each later pass combining with what is there (sum of per-pass means, or max).
+    const int tok_per_pass = 256 / sp.G;
+    for (int tok0 = 0; tok0 < sp.M_max; tok0 += tok_per_pass) {
+        p.tok0 = tok0;
+        p.tok_n = sp.M_max - tok0 < tok_per_pass ? sp.M_max - tok0 : tok_per_pass;
+        p.accumulate = tok0 > 0;
+        p.n_cols = p.tok_n * sp.G <= 128 ? 128 : 256;  // accumulator columns, padded to whole 128-row Q tiles
+        if (sp.score_mode == 1)
+            scores_tc_kernel<true><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
+        else
+            scores_tc_kernel<false><<<grid, kScoreThreads, kScoreSmem, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+        count_launch();
+    }
     return SPECPV_OK;
 }
 

@@ -247,3 +247,37 @@ def test_verify_host_matches_the_device_call_and_the_oracle(name, L, over):
                                          wl.to_numpy(w.v_pool[l]), wl.to_numpy(w.block_table[b]), int(c["ctx"][b]))
     util.compare(out_h[l, b].numpy(), o_out, c["dtype"], "verify_host")
     np.testing.assert_allclose(lse_h[l, b].numpy(), o_lse, atol=5e-3)
+
+
+@pytest.mark.parametrize("score_mode", [0, 1])
+@pytest.mark.parametrize("reduce", [B.REDUCE_MEAN, B.REDUCE_MAX, B.REDUCE_LAST])
+def test_scores_of_a_refresh_step_with_more_rows_than_one_accumulator(reduce, score_mode):
+    """A refresh scores with the chain and the tree together: 90 and 77 tokens x 4 heads = 360 and 308 query rows per
+    KV head, which the tensor-core kernel takes in two passes of 64 tokens (the second sequence's second pass is
+    ragged); the "last" row sits in the second pass for one sequence and in the first for the other."""
+    w = wl.make_workload("llama_32k", device="cuda", n_layers=2, M=90, ctx=[64 * 140 + 9, 64 * 300 + 1])
+    c = w.cfg
+    Hkv, d, M, batch, L = c["Hkv"], c["d"], c["M"], w.batch, c["n_layers"]
+    cfg = util.config_for(w, reduce=reduce, score_mode=score_mode)
+    full = util.full_cache(w)
+    ws = B.new_workspace(cfg, L, batch, int(max(c["ctx"])), M)
+    kmax = torch.zeros((L, batch, Hkv, w.max_blocks, d), dtype=torch.bfloat16, device="cuda")
+    kmin = torch.zeros_like(kmax)
+    B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax, kmin, ws)
+    q_lens = torch.tensor([90, 77], dtype=torch.int32, device="cuda")
+    last = torch.tensor([71, 5], dtype=torch.int32, device="cuda")
+    scores = torch.full((L, batch, Hkv, w.max_blocks), float("nan"), dtype=torch.float32, device="cuda")
+    B.specpv_score_blocks(cfg, 0, L, w.q, q_lens, M, last, kmax, kmin, full, scores, ws)
+    util.sync_status(ws)
+    for l in range(L):
+        for b in range(batch):
+            sl = int(c["ctx"][b])
+            nb = (sl + c["bs"] - 1) // c["bs"]
+            okmax, okmin = oracle.block_summaries(wl.to_numpy(w.k_pool[l]), wl.to_numpy(w.block_table[b]), sl)
+            m = int(q_lens[b])
+            osc = oracle.block_scores(wl.to_numpy(w.q[l, b, :m]), okmax, okmin, Hkv, reduce=reduce, last_query=int(last[b]),
+                                      score_mode=score_mode)
+            got = scores[l, b, :, :nb].cpu().numpy().astype(np.float64)
+            assert np.isfinite(got).all()
+            np.testing.assert_allclose(got, osc, rtol=2e-3, atol=2e-2, err_msg=f"layer {l} seq {b}")
+            assert torch.isnan(scores[l, b, :, nb:]).all()  # blocks past the context are left alone
