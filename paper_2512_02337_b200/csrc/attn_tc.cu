@@ -667,7 +667,7 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
     const double t_tile = 1.3, t_cta = 6.0, t_partial = 3.0, t_merge_launch = 6.0;
     const double avg_tiles = max_tiles + 1.0;  // context tiles + the tile of the step's own tokens
     for (int s = 1; s <= 64; ++s) {
-        if (s > 1 && (s > max_tiles / 4 || per_split * s > a.partial_bytes)) break;
+        if (s > 1 && (s > max_tiles / 2 || per_split * s > a.partial_bytes)) break;  // at least two tiles per CTA
         const long long ctas = (long long)base * s;
         const double waves = (double)((ctas + 147) / 148);
         double cost = waves * (t_cta + t_tile * (avg_tiles / s + (s > 1 ? 0.5 : 0.0)));
