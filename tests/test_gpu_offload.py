@@ -38,7 +38,8 @@ def refresh_tail(cfg, w, cache, q, mask, accepted, n_accepted, A_max, kmax, kmin
     return scores, idx, count, pk, pv, plens
 
 
-@pytest.mark.parametrize("name,over,L", [("llama_32k", dict(ctx=[9000]), 5), ("tiny_fp32", dict(), 1),
+@pytest.mark.parametrize("name,over,L", [("llama_32k", dict(ctx=[9000]), 5), ("llama_32k", dict(ctx=[700]), 2),
+                                         ("tiny_fp32", dict(), 1),
                                          ("stress_b4", dict(ctx=[3000, 4100, 2000, 3900]), 3)])
 def test_refresh_step_with_the_full_cache_in_host_memory(name, over, L):
     w = wl.make_workload(name, device="cuda", n_layers=L, spare_tokens=128, **over)

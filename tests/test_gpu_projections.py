@@ -70,6 +70,8 @@ CASES = [
     ("bf16", 8, 2, 128, 448, 1, 37, 3, 1, 2),       # seven 64-wide input steps over seven ranges, layers 1-2 of 3
     ("bf16", 8, 4, 128, 1024, 4, 64, 10, 0, 10),    # 160 tiles: one range per tile, 256 rows per tile
     ("bf16", 4, 2, 128, 256, 5, 64, 1, 0, 1),       # 320 rows: two row chunks
+    ("bf16", 2, 2, 128, 64, 1, 1, 1, 0, 1),         # one row, one 64-wide input step, no grouping of heads
+    ("bf16", 16, 2, 128, 2048, 3, 43, 2, 0, 2),     # 129 rows: the 128-row staging limit is passed by one
 ]
 
 
