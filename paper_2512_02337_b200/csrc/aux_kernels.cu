@@ -393,7 +393,22 @@ __global__ void __launch_bounds__(128) gather_kernel(GatherParams p) {
     const uint4* vs = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(p.full_v) + src_off);
     uint4* kd = reinterpret_cast<uint4*>(reinterpret_cast<char*>(p.part_k) + dst_off);
     uint4* vd = reinterpret_cast<uint4*>(reinterpret_cast<char*>(p.part_v) + dst_off);
-    for (size_t i = threadIdx.x; i < n_vec; i += blockDim.x) {
+    // four 16-byte loads of K and of V in flight per thread before the stores
+    size_t i = threadIdx.x;
+    for (; i + 3 * blockDim.x < n_vec; i += 4 * blockDim.x) {
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            a[u] = __ldg(ks + i + u * blockDim.x);
+            b[u] = __ldg(vs + i + u * blockDim.x);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            kd[i + u * blockDim.x] = a[u];
+            vd[i + u * blockDim.x] = b[u];
+        }
+    }
+    for (; i < n_vec; i += blockDim.x) {
         kd[i] = ks[i];
         vd[i] = vs[i];
     }
