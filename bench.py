@@ -600,21 +600,22 @@ def main():
         ms_step, e2e_max = max_over_ranks([ms_step, e2e_ms if not args.no_e2e else 0.0], dev)
         if not args.no_e2e:
             e2e_ms = e2e_max
-    sweep = None
-    if not args.no_sweep and rank == 0 and args.budget_blocks is None and args.block_tokens is None and c["dtype"] == "bf16":
-        sweep = partial_budget_sweep(st, load_peaks())
-    graph_times = None
-    if not args.no_graph and rank == 0 and c["dtype"] == "bf16":
-        graph_times = per_layer_graph(st)
-    block = None
-    if not args.no_block and rank == 0 and c["dtype"] == "bf16":
-        block = attention_block(st, load_peaks())
-    variants = None
-    if not args.no_sweep and rank == 0 and c["dtype"] == "bf16":
-        variants = score_variants(st, load_peaks())
-    offload = None
-    if not args.no_offload and rank == 0 and c["dtype"] == "bf16":
-        offload = offloaded_refresh(st)
+    # The side measurements below never take the headline line down with them: one that fails (for instance no room for
+    # the page-locked host copy of four layers) reports its error text in its place.
+    def side(enabled, fn, *fn_args):
+        if not (enabled and rank == 0 and c["dtype"] == "bf16"):
+            return None
+        try:
+            return fn(*fn_args)
+        except Exception as exc:  # noqa: BLE001
+            torch.cuda.synchronize(dev)
+            return {"error": f"{type(exc).__name__}: {exc}"[:300]}
+    sweep = side(not args.no_sweep and args.budget_blocks is None and args.block_tokens is None, partial_budget_sweep, st,
+                 load_peaks())
+    graph_times = side(not args.no_graph, per_layer_graph, st)
+    block = side(not args.no_block, attention_block, st, load_peaks())
+    variants = side(not args.no_sweep, score_variants, st, load_peaks())
+    offload = side(not args.no_offload, offloaded_refresh, st)
     if rank != 0:
         return 0
 
