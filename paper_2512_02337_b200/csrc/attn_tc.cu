@@ -572,18 +572,33 @@ __global__ void __launch_bounds__(32 * kMergeRows) merge_tc_kernel(TcParams p) {
     for (int s = 0; s < p.n_splits; ++s) m_all = fmaxf(m_all, ml[(base + s) * p.R_pad + r].x);
     float l_all = 0.f;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int s = 0; s < p.n_splits; ++s) {
-        const size_t prow = (base + s) * p.R_pad + r;
-        const float2 m_l = ml[prow];
-        if (m_l.x == -INFINITY) continue;  // an empty split: its partial O was never written
-        const float4 po = reinterpret_cast<const float4*>(p.part_o + prow * kD)[lane];
-        const float w = __expf(m_l.x - m_all);
-        l_all = fmaf(m_l.y, w, l_all);
-        o.x = fmaf(po.x, w, o.x);
-        o.y = fmaf(po.y, w, o.y);
-        o.z = fmaf(po.z, w, o.z);
-        o.w = fmaf(po.w, w, o.w);
+    // four splits at a time, their loads in flight together (added in split order, so the result does not depend on
+    // the batching); an empty split's partial O was never written and is not read
+    for (int s0 = 0; s0 < p.n_splits; s0 += 4) {
+        float2 m_l[4];
+        float4 po[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t prow = (base + min(s0 + u, p.n_splits - 1)) * p.R_pad + r;
+            m_l[u] = ml[prow];
+            if (s0 + u >= p.n_splits) m_l[u].x = -INFINITY;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t prow = (base + min(s0 + u, p.n_splits - 1)) * p.R_pad + r;
+            po[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (m_l[u].x != -INFINITY) po[u] = __ldg(reinterpret_cast<const float4*>(p.part_o + prow * kD) + lane);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (m_l[u].x == -INFINITY) continue;
+            const float w = __expf(m_l[u].x - m_all);
+            l_all = fmaf(m_l[u].y, w, l_all);
+            o.x = fmaf(po[u].x, w, o.x);
+            o.y = fmaf(po[u].y, w, o.y);
+            o.z = fmaf(po[u].z, w, o.z);
+            o.w = fmaf(po[u].w, w, o.w);
+        }
     }
     const int j = r / p.G, g = r % p.G;
     const size_t row = ((size_t)lb * p.M_max + j) * p.Hq + h * p.G + g;
