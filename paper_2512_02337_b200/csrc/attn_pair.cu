@@ -1,0 +1,667 @@
+// Tensor-core verification attention on CTA pairs (B200, sm_100a): bfloat16, head_dim 128, pages of 16, 32 or 64
+// tokens, more than 128 query rows per KV head.  Tree-masked GQA attention of the step's tokens over a paged cache
+// (paper Section 3.2-3.3, Algorithm 1 "TreeDecode"), for both the partial and the full cache.
+//
+// A cluster of two CTAs owns one (layer, sequence, KV head, KV split, group of 256 rows).  Each CTA holds one
+// 128-row tile of the group (row = step token * G + query head) and HALF of every 128-token K/V tile: the 64 tokens
+// of K it contributes to S = Q K^T and the 64 channels of V it contributes to O += P V.  The contractions are
+// pair-wide tcgen05.mma (cta_group::2, M = 256), issued by one thread of the even CTA, which read both CTAs'
+// shared memory, so a K/V byte is fetched from HBM once and read from shared memory once per pair.
+//
+// Work is organised in steps: step t loads K of tile t and V of tile t-3 into ring slot t % 5 and issues
+// PV(t-3) then QK(t).  S lives in one of THREE tensor-memory buffers (tile mod 3) and P(j) overwrites the first
+// half of S(j)'s own buffer, so that the softmax warps never wait for a buffer: the buffer of tile j is theirs from
+// the completion of QK(j) until they hand P(j) over, and QK(j+3), which reuses it, is issued behind PV(j) on the
+// in-order tensor pipe.  The only wait on the critical loop is the issuer's wait for P(j).
+//   warp 0      TMA producer (both CTAs): its Q tile per stretch, then per step its K and V halves through the block
+//               table (128-byte swizzle); completion is counted on the even CTA's barriers
+//   warp 1      MMA issuer (even CTA): per step  PV(t-3), QK(t), two commits (S ready; step done = slot free)
+//   warp 2      zeroes the rows of its V half past the valid tokens (ragged last tile, the step's own tokens)
+//   warps 4-11  softmax (both CTAs): a warp owns 16 rows, four threads per row (tcgen05.ld 16x256b), so the row
+//               maximum and the overflow check stay inside the warp; online softmax in the log2 domain with a
+//               reference maximum that is only moved when it must be
+// Tensor memory (512 columns per CTA): S0/P0 | S1/P1 | S2/P2 | O (128 columns each).
+// With several KV splits the unnormalised (O, m, l) go to the workspace and the merge kernel combines them by
+// log-sum-exp.  Every wait is bounded; a wait that gives up records SPECPV_ERR_TIMEOUT, stops its loop, raises
+// the abort flag of both CTAs, and the pair still drains its copies and frees its tensor memory.
+#include "attn_tc.cuh"
+
+namespace specpv {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kPairThreads = 384;   // 12 warps
+constexpr int kRing = 5;            // steps in flight per CTA
+constexpr int kSlot = 32768;        // [K half of tile t: 2 d-halves x 64 tokens x 64 d][V half of tile t-3: 128 tokens x 64 channels]
+constexpr int kVOff = 16384;
+constexpr int kQTile = 32768;       // [2 d-halves][128 rows][64 d]
+constexpr int kPairSmem = 1024 + 2 * kQTile + kRing * kSlot;
+constexpr uint32_t kColO = 384;     // tensor-memory columns: S/P buffer b at b * 128, O behind them
+constexpr int kLag = 3;             // PV runs this many tiles behind QK (= number of S/P buffers)
+constexpr uint64_t kWaitNs = 2000000000ull;
+
+// Instruction descriptors, kind::f16: D = f32, A = B = bf16, M = 256 over the pair, N = 128.
+constexpr uint32_t idesc_pair(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
+}
+constexpr uint32_t kIdescQK2 = idesc_pair(false);
+constexpr uint32_t kIdescPV2 = idesc_pair(true);  // B (= V) is MN-major
+
+struct __align__(8) PairBars {
+    uint64_t q_full[2];          // even CTA: both CTAs' Q tiles of a stretch have landed (transaction bytes)
+    uint64_t q_empty[2];         // both: the last QK of the stretch that used this Q buffer has completed
+    uint64_t ld_full[kRing];     // even CTA: a step's K and V halves are in place (bytes + one "V ready" per CTA)
+    uint64_t step_done[kRing];   // both: the step's PV and QK have completed (its slot is free; O holds that PV)
+    uint64_t vfix_full[kRing];   // own: this CTA's V half of a tile that needs zeroed rows has landed
+    uint64_t s_full[kLag];       // both: S(j) is complete
+    uint64_t p_full[kLag];       // even CTA: all 16 softmax warps have stored P(j)
+    uint64_t o_full;             // both: the last PV of a stretch has completed
+    uint64_t o_free;             // even CTA: all 16 softmax warps have read O of the finished stretch
+    uint64_t drain;              // even CTA: completion of whatever was issued before an abort
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// One stretch of KV tiles of one (layer, sequence, KV head, row group) processed by a pair.
+struct Seg {
+    int lb, b, l, h, rg, split;
+    int M, seq_len, tok0;
+    int tile_begin;   // first context tile (128 tokens each) of the stretch
+    int n_ctx;        // context tiles in the stretch
+    int n_tiles;      // n_ctx + 1 if the stretch ends with the tile of the step's own tokens
+    int first_fix;    // first tile (stretch-local) whose V rows past the valid tokens must be zeroed; n_tiles if none
+    bool direct;      // the stretch covers the whole KV range: results are final
+};
+
+// The stretches of a pair, in order.  Here: exactly one, given by the grid position.
+struct SegIter {
+    bool done = false;
+    __device__ bool next(const TcParams& p, Seg& s) {
+        if (done) return false;
+        done = true;
+        const int pair_x = blockIdx.x >> 1;
+        s.split = pair_x % p.n_splits;
+        s.rg = pair_x / p.n_splits;
+        s.h = blockIdx.y;
+        s.lb = blockIdx.z;
+        s.b = s.lb % p.batch;
+        s.l = s.lb / p.batch;
+        s.seq_len = max(p.seq_lens[s.b], 0);
+        int M = p.q_lens ? p.q_lens[s.b] : p.M_max;
+        s.M = min(max(M, 0), p.M_max);
+        s.tok0 = s.rg * (256 / p.G);
+        const int total_tiles = (s.seq_len + kTileTokens - 1) / kTileTokens;
+        const int tiles_per_split = (total_tiles + p.n_splits - 1) / p.n_splits;
+        s.tile_begin = min(s.split * tiles_per_split, total_tiles);
+        const int tile_end = min(s.tile_begin + tiles_per_split, total_tiles);
+        const bool last_split = s.split == p.n_splits - 1;
+        s.n_ctx = tile_end - s.tile_begin;
+        s.n_tiles = s.n_ctx + (last_split ? 1 : 0);
+        const bool ragged_ctx = s.n_ctx > 0 && tile_end == total_tiles && (s.seq_len % kTileTokens) != 0;
+        s.first_fix = ragged_ctx ? s.n_ctx - 1 : ((last_split && s.M < kTileTokens) ? s.n_ctx : s.n_tiles);
+        s.direct = p.n_splits == 1;
+        return true;
+    }
+};
+
+// Bounded wait for the pair kernel: a wait that gives up records the fault and raises the abort flag of both CTAs.
+__device__ __forceinline__ bool pair_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
+                                               void* workspace, int where, uint64_t limit_ns) {
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((it & 255u) == 255u && global_ns() - t0 > limit_ns) {
+            *abort_flag = 1;
+            st_cluster_u32(peer_abort, 1u);
+            record_fault(workspace, SPECPV_ERR_TIMEOUT, where, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool pair_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
+                                          void* workspace, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return pair_wait_slow(bar, parity, abort_flag, peer_abort, workspace, where, kWaitNs);
+}
+
+// =================================================================================================
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) attn_pair_kernel(const __grid_constant__ TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the 128-byte swizzle atoms (the same offset in both CTAs)
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ PairBars bars;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: the CTA that issues the contractions and counts the completions
+    const int tok_per_tile = 128 / p.G;       // step tokens per 128-row tile
+
+    // Uniform early exits (both CTAs of a pair see the same stretch).
+    {
+        SegIter it;
+        Seg s;
+        it.next(p, s);
+        if (s.tok0 >= s.M) return;
+        if (s.n_tiles == 0) {
+            // an empty split: publish (m = -inf, l = 0) so that the merge ignores it
+            for (int r = threadIdx.x; r < 128; r += kPairThreads) {
+                const int row = s.rg * 256 + (int)rank * 128 + r;
+                const size_t prow = (((size_t)s.lb * p.Hkv + s.h) * p.n_splits + s.split) * p.R_pad + row;
+                p.part_ml[prow * 2] = -INFINITY;
+                p.part_ml[prow * 2 + 1] = 0.f;
+            }
+            return;
+        }
+    }
+
+    const uint32_t q_smem = smem_u32(smem);
+    const uint32_t kv_smem = q_smem + 2 * kQTile;
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t peer_abort = mapa(smem_u32(&bars.abort_flag), rank ^ 1u);
+
+    // ---- set-up ------------------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&bars.q_full[i]), 1);
+            mbar_init(smem_u32(&bars.q_empty[i]), 1);
+        }
+        for (int i = 0; i < kLag; ++i) {
+            mbar_init(smem_u32(&bars.s_full[i]), 1);
+            mbar_init(smem_u32(&bars.p_full[i]), 16);  // one arrival per softmax warp of the pair
+        }
+        for (int s = 0; s < kRing; ++s) {
+            mbar_init(smem_u32(&bars.ld_full[s]), 3);  // the byte count's arrival + one "V half ready" per CTA
+            mbar_init(smem_u32(&bars.step_done[s]), 1);
+            mbar_init(smem_u32(&bars.vfix_full[s]), 1);
+        }
+        mbar_init(smem_u32(&bars.o_full), 1);
+        mbar_init(smem_u32(&bars.o_free), 16);
+        mbar_init(smem_u32(&bars.drain), 1);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {  // one warp of each CTA: the allocation is made in both CTAs' tensor memory at once
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&bars.tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem = bars.tmem_base;
+
+    // barriers of the even CTA, as seen from this CTA
+    const uint32_t lead_q_full0 = mapa(smem_u32(&bars.q_full[0]), 0);
+    const uint32_t lead_ld_full0 = mapa(smem_u32(&bars.ld_full[0]), 0);
+    const uint32_t lead_p_full0 = mapa(smem_u32(&bars.p_full[0]), 0);
+    const uint32_t lead_o_free = mapa(smem_u32(&bars.o_free), 0);
+
+    // Register budget: the control warpgroup (warps 0-3) gives registers to the two softmax warpgroups.
+    if (warp == 0) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // =========================== TMA producer ================================================
+        // The whole warp runs the loop; lane 0 does the barrier bookkeeping, each copy is issued by its own lane.
+        // Step t brings K of tile t (stretch walker `k`) and V of tile t - 3 (walker `v`) into slot t % 5.
+        const int ppt = kTileTokens / p.bs;  // pages per tile
+        // K copies: lane 2 pg + half, pg < ppt / 2 (this CTA's 64 tokens), half = 64-channel half of d
+        // V copies: lane 16 + pg, pg < ppt (all 128 tokens, this CTA's 64 channels)
+        const bool k_lane = lane < ppt, v_lane = lane >= 16 && lane < 16 + ppt;
+        const int k_pg = lane >> 1, k_half = lane & 1, v_pg = lane - 16;
+        SegIter it_k, it_v;
+        Seg sk, sv;
+        bool have_k = it_k.next(p, sk), have_v = it_v.next(p, sv);
+        int jk = 0, jv = 0, sidx_k = 0;
+        bool ok = true;
+        // pool row of this lane's page of context tile j of a stretch (an out-of-range row makes the copy engine fill zeros)
+        auto page_row = [&](const Seg& s, int j, bool is_k) {
+            int row = (int)p.pool_rows;
+            const int blk = (s.tile_begin + j) * ppt + (is_k ? (int)rank * (ppt >> 1) + k_pg : v_pg);
+            if ((long long)blk * p.bs < s.seq_len && blk < p.max_blocks) {
+                const int page = p.block_table[(size_t)s.b * p.max_blocks + blk];
+                if (page < 0 || page >= p.n_pages) {
+                    if (is_k ? k_half == 0 : rank == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, s.b, blk, page, s.l);
+                } else {
+                    row = (int)((((long long)(p.layer0 + s.l) * p.n_pages + page) * p.Hkv + s.h) * p.bs);
+                }
+            }
+            return row;
+        };
+        for (uint32_t t = 0; ok && (have_k || have_v); ++t) {
+            if (have_k && jk == 0) {  // the stretch's Q tile, ahead of its first K tile
+                const int qb = sidx_k & 1;
+                if (sidx_k >= 2) ok = pair_wait(smem_u32(&bars.q_empty[qb]), ((sidx_k >> 1) - 1) & 1, abort_flag, peer_abort, p.workspace, 1);
+                if (!ok) break;
+                if (lane == 0) {
+                    if (rank == 0) mbar_expect_tx(smem_u32(&bars.q_full[qb]), 2 * kQTile);
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_3d_pair(q_smem + qb * kQTile + half * 16384, &p.tm_q, half * 64, sk.h * p.G,
+                                         sk.lb * p.M_max + sk.tok0 + (int)rank * tok_per_tile, lead_q_full0 + qb * 8);
+                }
+                __syncwarp();
+            }
+            const uint32_t slot = t % kRing;
+            const bool do_v = have_v && t >= (uint32_t)kLag;
+            const bool fix = do_v && jv >= sv.first_fix;
+            int row_mine = (int)p.pool_rows;
+            if (k_lane && have_k && jk < sk.n_ctx) row_mine = page_row(sk, jk, true);
+            if (v_lane && do_v && jv < sv.n_ctx) row_mine = page_row(sv, jv, false);
+            if (t >= (uint32_t)kRing) ok = pair_wait(smem_u32(&bars.step_done[slot]), ((t / kRing) - 1) & 1, abort_flag, peer_abort, p.workspace, 2);
+            if (!ok) break;
+            const uint32_t slot_base = kv_smem + slot * kSlot;
+            const uint32_t full = lead_ld_full0 + slot * 8, vfix = smem_u32(&bars.vfix_full[slot]);
+            if (lane == 0) {
+                if (rank == 0) mbar_expect_tx(smem_u32(&bars.ld_full[slot]), (have_k ? kSlot : 0) + ((do_v && !fix) ? kSlot : 0));
+                if (fix) mbar_expect_tx(vfix, kSlot - kVOff);
+            }
+            __syncwarp();
+            if (have_k) {
+                if (jk >= sk.n_ctx) {  // the step's own tokens
+                    if (lane < 2)
+                        tma_load_3d_pair(slot_base + lane * 8192, &p.tm_knew, lane * 64, sk.h, sk.lb * p.M_max + (int)rank * 64, full);
+                } else if (k_lane) {
+                    tma_load_2d_pair(slot_base + k_half * 8192 + k_pg * p.bs * 128, &p.tm_kpool, k_half * 64, row_mine, full);
+                }
+            }
+            if (do_v) {
+                const uint32_t vbar = fix ? vfix : full;
+                if (jv >= sv.n_ctx) {
+                    if (lane == 16 || lane == 17)
+                        tma_load_3d_pair(slot_base + kVOff + (lane - 16) * 8192, &p.tm_vnew, (int)rank * 64, sv.h,
+                                         sv.lb * p.M_max + (lane - 16) * 64, vbar);
+                } else if (v_lane) {
+                    tma_load_2d_pair(slot_base + kVOff + v_pg * p.bs * 128, &p.tm_vpool, (int)rank * 64, row_mine, vbar);
+                }
+            }
+            __syncwarp();
+            if (lane == 0 && !fix) mbar_arrive_cluster(full);  // this CTA's V half needs no zeroing (or the step has none)
+            if (have_k && ++jk == sk.n_tiles) { have_k = it_k.next(p, sk); jk = 0; ++sidx_k; }
+            if (do_v && ++jv == sv.n_tiles) { have_v = it_v.next(p, sv); jv = 0; }
+        }
+    } else if (warp == 1) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // =========================== MMA issuer (even CTA) =======================================
+        // One thread issues every contraction of the pair: per step  PV(t-3), QK(t).  PV(t-3) reads P from the
+        // buffer that QK(t) overwrites; the tensor pipe runs in order, so no wait lies between them.  The step and
+        // tile counters run across stretches, so the pipeline does not drain between them; only O is handed over.
+        if (rank == 0) {
+            const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
+            const uint32_t q_lo0 = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            const uint32_t k_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            const uint32_t v_lo0 = (((kv_smem + kVOff) >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            SegIter it_k, it_v;  // it_k walks the QK side, it_v the PV side
+            Seg sk, sv;
+            bool have_k = it_k.next(p, sk), have_v = it_v.next(p, sv);
+            int jk = 0, jv = 0, sidx_k = 0, sidx_v = 0;
+            bool ok = true;
+            for (uint32_t t = 0; ok && (have_k || have_v); ++t) {
+                const uint32_t slot = t % kRing, buf = t % kLag;
+                const bool do_v = have_v && t >= (uint32_t)kLag;
+                if (have_k && jk == 0) ok = pair_wait(smem_u32(&bars.q_full[sidx_k & 1]), (sidx_k >> 1) & 1, abort_flag, peer_abort, p.workspace, 3);
+                if (ok) ok = pair_wait(smem_u32(&bars.ld_full[slot]), (t / kRing) & 1, abort_flag, peer_abort, p.workspace, 4);
+                if (ok && do_v) {
+                    if (jv == 0 && sidx_v > 0) ok = pair_wait(smem_u32(&bars.o_free), (sidx_v - 1) & 1, abort_flag, peer_abort, p.workspace, 6);
+                    if (ok) ok = pair_wait(smem_u32(&bars.p_full[buf]), ((t - kLag) / kLag) & 1, abort_flag, peer_abort, p.workspace, 7);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    if (do_v) {  // O += P(t-3) V
+                        const uint32_t b_lo = launder(v_lo0 + slot * (kSlot >> 4));
+                        const uint32_t a = tmem + buf * 128, d = tmem + kColO;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)  // 16 tokens per instruction: two 8-row groups of 1024 bytes
+                            mma2_ts_lohi(d, a + kk * 8, b_lo + (uint32_t)kk * (2048u >> 4), desc_hi, kIdescPV2, (jv > 0 || kk > 0) ? 1u : 0u);
+                        if (jv == sv.n_tiles - 1) tc_commit_pair(smem_u32(&bars.o_full));
+                    }
+                    if (have_k) {  // S(t) = Q K^T
+                        const uint32_t a_lo = launder(q_lo0 + (uint32_t)(sidx_k & 1) * (kQTile >> 4));
+                        const uint32_t b_lo = launder(k_lo0 + slot * (kSlot >> 4));
+                        const uint32_t d = tmem + buf * 128;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
+                            const uint32_t a_off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                            const uint32_t b_off = (uint32_t)((kk >> 2) * 8192 + (kk & 3) * 32) >> 4;
+                            mma2_ss_lohi(d, a_lo + a_off, b_lo + b_off, desc_hi, kIdescQK2, kk > 0 ? 1u : 0u);
+                        }
+                        tc_commit_pair(smem_u32(&bars.s_full[buf]));
+                        if (jk == sk.n_tiles - 1) tc_commit_pair(smem_u32(&bars.q_empty[sidx_k & 1]));
+                    }
+                    tc_commit_pair(smem_u32(&bars.step_done[slot]));
+                }
+                __syncwarp();
+                if (have_k && ++jk == sk.n_tiles) { have_k = it_k.next(p, sk); jk = 0; ++sidx_k; }
+                if (do_v && ++jv == sv.n_tiles) { have_v = it_v.next(p, sv); jv = 0; ++sidx_v; }
+            }
+        }
+    } else if (warp == 2) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // =========================== V fixer =====================================================
+        // Rows of a V tile past its valid tokens may hold anything (stale pages, rows of other sequences' steps): zero
+        // them in this CTA's half so that 0 * garbage cannot give NaN, then report the half ready.  Only a ragged last
+        // context tile and the tile of the step's own tokens need it; their V copies complete on this CTA's own barrier.
+        SegIter it;
+        Seg s;
+        uint32_t g = 0, fix_parity = 0;  // bit `slot`: parity of the next fix use of that slot's barrier
+        bool ok = true;
+        while (ok && it.next(p, s)) {
+            for (int j = s.first_fix; j < s.n_tiles; ++j) {
+                const uint32_t slot = (g + j + kLag) % kRing;  // V of tile g + j travels with step g + j + 3
+                ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.vfix_full[slot]), (fix_parity >> slot) & 1u, abort_flag,
+                                                       peer_abort, p.workspace, 8));
+                if (!ok) break;
+                fix_parity ^= 1u << slot;
+                const int n_valid = j >= s.n_ctx ? s.M : min(kTileTokens, s.seq_len - (s.tile_begin + j) * kTileTokens);
+                uint8_t* v = smem + 2 * kQTile + (size_t)slot * kSlot + kVOff;
+                const int n_rows = kTileTokens - max(n_valid, 0);
+                for (int i = lane; i < n_rows * 8; i += 32)
+                    *reinterpret_cast<uint4*>(v + (size_t)(max(n_valid, 0) + (i >> 3)) * 128 + (i & 7) * 16) = make_uint4(0, 0, 0, 0);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(lead_ld_full0 + slot * 8);
+            }
+            g += (uint32_t)s.n_tiles;
+        }
+    } else if (warp == 3) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        // =========================== softmax / correction / epilogue ==============================
+        const int q = warp & 3;                    // tensor-memory lane quarter this warp may access
+        const int hf = (warp - 4) >> 2;            // lower or upper 16 lanes of the quarter
+        const int lrow = q * 32 + hf * 16;
+        const int ra = lrow + (lane >> 2), rb = ra + 8;   // this thread's two rows within the CTA's tile
+        const int cq = (lane & 3) * 2;             // its two adjacent columns in every group of eight
+        const uint32_t lane_addr = (uint32_t)lrow << 16;
+        const uint32_t o_addr = tmem + lane_addr + kColO;
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+        SegIter it;
+        Seg s;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+            const int row_a = (int)rank * 128 + ra, row_b = (int)rank * 128 + rb;  // rows within the row group
+            const int tok_a = s.tok0 + row_a / p.G, tok_b = s.tok0 + row_b / p.G;
+            const bool valid_a = tok_a < s.M, valid_b = tok_b < s.M;
+            uint64_t mlo_a = 0, mhi_a = 0, mlo_b = 0, mhi_b = 0;
+            if (valid_a) {
+                const uint64_t* mrow = p.tree_mask + ((size_t)s.b * p.M_max + tok_a) * p.mask_words;
+                mlo_a = mrow[0];
+                if (p.mask_words > 1) mhi_a = mrow[1];
+            }
+            if (valid_b) {
+                const uint64_t* mrow = p.tree_mask + ((size_t)s.b * p.M_max + tok_b) * p.mask_words;
+                mlo_b = mrow[0];
+                if (p.mask_words > 1) mhi_b = mrow[1];
+            }
+            float m_a = -INFINITY, m_b = -INFINITY;  // reference maxima (log2 domain), the same in the four threads of a row
+            float l_a = 0.f, l_b = 0.f;              // this thread's share of the row sums
+            for (int j = 0; j < s.n_tiles && ok; ++j, ++g) {
+                const bool is_new = j >= s.n_ctx;
+                const int n_valid = is_new ? s.M : min(kTileTokens, s.seq_len - (s.tile_begin + j) * kTileTokens);
+                const bool masked = is_new || n_valid < kTileTokens;
+                const uint32_t buf = g % kLag;
+                const uint32_t s_addr = tmem + lane_addr + buf * 128;
+                ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.s_full[buf]), (g / kLag) & 1, abort_flag, peer_abort, p.workspace, 9));
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t v[64];  // v[4n + k]: row a (k < 2) or b, column 8n + cq + (k & 1)
+                TMEM_LD_16x256_X8(s_addr, v);
+                TMEM_LD_16x256_X8(s_addr + 64, (v + 32));
+                tmem_wait_ld();
+                // P = 2^(s*scale - m) as bf16 pairs: word 2n + k/2 of P (row a or b, columns 8n + cq, + 1) goes to
+                // v[2n + k/2], whose own value was consumed earlier.  The row sums are taken over the ROUNDED weights
+                // the tensor core will use, so that O / l is an exact weighted average of V rows.
+                auto exp_rows = [&](float ma, float mb, float& sum_a, float& sum_b) {
+                    const float2 na = make_float2(-ma, -ma), nb = make_float2(-mb, -mb);
+                    float2 acc_a[2], acc_b[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) acc_a[e] = acc_b[e] = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int n = 0; n < 16; ++n) {
+                        const float2 xa = __ffma2_rn(make_float2(__uint_as_float(v[4 * n]), __uint_as_float(v[4 * n + 1])), sc2, na);
+                        const float2 xb = __ffma2_rn(make_float2(__uint_as_float(v[4 * n + 2]), __uint_as_float(v[4 * n + 3])), sc2, nb);
+                        const uint32_t wa = pack_bf16(ex2(xa.x), ex2(xa.y));
+                        const uint32_t wb = pack_bf16(ex2(xb.x), ex2(xb.y));
+                        v[2 * n] = wa;
+                        v[2 * n + 1] = wb;
+                        add_bf16_pair(acc_a[n & 1], wa);
+                        add_bf16_pair(acc_b[n & 1], wb);
+                    }
+                    sum_a = (acc_a[0].x + acc_a[1].x) + (acc_a[0].y + acc_a[1].y);
+                    sum_b = (acc_b[0].x + acc_b[1].x) + (acc_b[0].y + acc_b[1].y);
+                };
+                // Fast path (every full context tile after the first of a stretch): keep the reference maxima and skip
+                // the row maximum.  Weights may then exceed 1; float32 sums and bf16 weights keep their relative precision
+                // whatever the exponent, so only overflow has to be ruled out: if a row's share of the sum leaves the safe
+                // range (or a row has no reference yet), the warp takes the tile again from tensor memory (S(j) stays
+                // intact until every warp has arrived on the P barrier) on the general path.
+                float add_a = 0.f, add_b = 0.f;
+                bool general = j == 0 || masked;
+                if (!general) {
+                    exp_rows(m_a, m_b, add_a, add_b);
+                    const bool bad = (valid_a && (!(add_a < kSafeRowSum) || m_a == -INFINITY)) ||
+                                     (valid_b && (!(add_b < kSafeRowSum) || m_b == -INFINITY));
+                    if (__any_sync(0xffffffffu, bad)) {
+                        general = true;
+                        TMEM_LD_16x256_X8(s_addr, v);
+                        TMEM_LD_16x256_X8(s_addr + 64, (v + 32));
+                        tmem_wait_ld();
+                    }
+                }
+                if (general) {
+                    if (masked) {  // ragged or tree-masked tile: invisible columns become -inf
+                        uint64_t va_lo = ~0ull, va_hi = ~0ull, vb_lo = ~0ull, vb_hi = ~0ull;
+                        if (is_new) { va_lo = mlo_a; va_hi = mhi_a; vb_lo = mlo_b; vb_hi = mhi_b; }
+                        uint64_t keep_lo = ~0ull, keep_hi = ~0ull;
+                        if (n_valid < 64) {
+                            keep_lo = (n_valid <= 0) ? 0ull : (~0ull >> (64 - n_valid));
+                            keep_hi = 0;
+                        } else if (n_valid < 128) {
+                            keep_hi = (n_valid == 64) ? 0ull : (~0ull >> (128 - n_valid));
+                        }
+                        va_lo = (va_lo & keep_lo) >> cq; va_hi = (va_hi & keep_hi) >> cq;
+                        vb_lo = (vb_lo & keep_lo) >> cq; vb_hi = (vb_hi & keep_hi) >> cq;
+#pragma unroll
+                        for (int n = 0; n < 16; ++n) {
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint64_t word = (k < 2) ? (n < 8 ? va_lo : va_hi) : (n < 8 ? vb_lo : vb_hi);
+                                if (!((word >> ((n & 7) * 8 + (k & 1))) & 1ull)) v[4 * n + k] = 0xff800000u;
+                            }
+                        }
+                    }
+                    float xa0 = __uint_as_float(v[0]), xa1 = __uint_as_float(v[1]);
+                    float xb0 = __uint_as_float(v[2]), xb1 = __uint_as_float(v[3]);
+#pragma unroll
+                    for (int n = 1; n < 16; n += 2) {  // three-input max: two new values per instruction
+                        xa0 = fmax3(xa0, __uint_as_float(v[4 * n]), __uint_as_float(v[4 * n + 1]));
+                        xb0 = fmax3(xb0, __uint_as_float(v[4 * n + 2]), __uint_as_float(v[4 * n + 3]));
+                        if (n + 1 < 16) {
+                            xa1 = fmax3(xa1, __uint_as_float(v[4 * n + 4]), __uint_as_float(v[4 * n + 5]));
+                            xb1 = fmax3(xb1, __uint_as_float(v[4 * n + 6]), __uint_as_float(v[4 * n + 7]));
+                        }
+                    }
+                    float mx_a = fmaxf(xa0, xa1), mx_b = fmaxf(xb0, xb1);
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+                    const float mt_a = mx_a * p.scale_log2, mt_b = mx_b * p.scale_log2;
+                    // lazy rescale: keep the old reference unless the new maximum is more than 2^8 larger.  The decision
+                    // is per row, the tensor-memory traffic is warp-wide (factor 1 where nothing changes).
+                    bool need_a = false, need_b = false;
+                    if (j == 0) {
+                        m_a = mt_a;
+                        m_b = mt_b;
+                    } else {
+                        need_a = mt_a > m_a + kRescaleThreshold || (m_a == -INFINITY && mt_a > -INFINITY);
+                        need_b = mt_b > m_b + kRescaleThreshold || (m_b == -INFINITY && mt_b > -INFINITY);
+                    }
+                    if (__any_sync(0xffffffffu, need_a || need_b)) {
+                        const float fa = !need_a ? 1.f : (m_a == -INFINITY ? 0.f : ex2(m_a - mt_a));
+                        const float fb = !need_b ? 1.f : (m_b == -INFINITY ? 0.f : ex2(m_b - mt_b));
+                        // O must hold PV(j-1) before it is rescaled: that is step j+2, whose commit frees its slot (the
+                        // barrier cannot run a phase ahead: that takes PV(j+4), which needs the P this warp has not stored)
+                        ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.step_done[(g + 2) % kRing]), ((g + 2) / kRing) & 1,
+                                                               abort_flag, peer_abort, p.workspace, 10));
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            TMEM_LD_16x256_X8(o_addr + c * 64, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * ((i & 2) ? fb : fa));
+                            TMEM_ST_16x256_X8(o_addr + c * 64, o);
+                        }
+                        if (need_a) { l_a *= fa; m_a = mt_a; }
+                        if (need_b) { l_b *= fb; m_b = mt_b; }
+                    }
+                    exp_rows(m_a == -INFINITY ? 0.f : m_a, m_b == -INFINITY ? 0.f : m_b, add_a, add_b);
+                }
+                l_a += add_a;
+                l_b += add_b;
+                // P(j) goes over the first half of S(j)'s own buffer (nothing else touches it before PV(j))
+                TMEM_ST_16x128_X16(s_addr, v);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(lead_p_full0 + buf * 8);
+            }
+            if (!ok) break;
+            // ---- epilogue of the stretch: wait for the last PV, hand O back, normalise, write out ------------
+            ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.o_full), sidx & 1, abort_flag, peer_abort, p.workspace, 12));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t o[64];
+            TMEM_LD_16x256_X8(o_addr, o);
+            TMEM_LD_16x256_X8(o_addr + 64, (o + 32));
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(lead_o_free);
+            // the four threads of a row add their shares of the row sum
+            l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+            l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+            l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+            l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const bool valid = r ? valid_b : valid_a;
+                if (!valid) continue;
+                const int row = r ? row_b : row_a, tok = r ? tok_b : tok_a;
+                const float l_run = r ? l_b : l_a, m_run = r ? m_b : m_a;
+                const size_t out_row = ((size_t)s.lb * p.M_max + tok) * p.Hq + s.h * p.G + row % p.G;
+                const size_t prow = (((size_t)s.lb * p.Hkv + s.h) * p.n_splits + s.split) * p.R_pad + s.rg * 256 + row;
+                const float inv = s.direct ? 1.f / l_run : 1.f;
+#pragma unroll
+                for (int n = 0; n < 16; ++n) {
+                    const int ch = 8 * n + cq;
+                    const float x = __uint_as_float(o[4 * n + 2 * r]) * inv, y = __uint_as_float(o[4 * n + 2 * r + 1]) * inv;
+                    if (!s.direct) {
+                        *reinterpret_cast<float2*>(p.part_o + prow * kD + ch) = make_float2(x, y);
+                    } else if (p.out_f32) {
+                        *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.out) + out_row * kD + ch) = make_float2(x, y);
+                    } else {
+                        *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_row * kD + ch) = pack_bf16(x, y);
+                    }
+                }
+                if ((lane & 3) == 0) {
+                    if (s.direct) {
+                        if (p.lse) p.lse[out_row] = m_run * kLn2 + logf(l_run);
+                    } else {
+                        p.part_ml[prow * 2] = m_run * kLn2;  // natural-log units for the merge
+                        p.part_ml[prow * 2 + 1] = l_run;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----------------------------------------------------------------------------
+    // After an abort nothing new is issued; copies already in flight land within microseconds, contractions already
+    // issued are waited for (bounded) before the tensor memory goes back.
+    __syncwarp();
+    if (*abort_flag) {
+        __nanosleep(1000000);
+        if (warp == 1 && rank == 0) {
+            if (lane == 0) tc_commit_pair(smem_u32(&bars.drain));
+            __syncwarp();
+            const uint64_t t0 = global_ns();
+            while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < 100000000ull) {}
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA leaves while the other may still touch its shared memory or barriers
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+}  // namespace
+
+// The pair kernel serves the shapes of the single-CTA kernel whenever a KV head has more than one 128-row tile.
+bool attention_pair_wanted(const AttnArgs& a) { return a.M_max * a.g.G > 128; }
+
+specpv_status launch_attention_pair(TcParams& p, const AttnArgs& a, cudaStream_t stream) {
+    if (!set_smem_limit_once(reinterpret_cast<const void*>(attn_pair_kernel), kPairSmem)) return SPECPV_ERR_CUDA;
+    const int Hkv = a.g.Hkv;
+    const int R_max = a.M_max * a.g.G;
+    // KV splits: fill the pairs the device can hold at once (one CTA per SM) in whole waves
+    static int pairs_cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPECPV_ERR_CUDA;
+    int n_pairs = (dev >= 0 && dev < 64) ? pairs_cached[dev] : 0;
+    if (n_pairs <= 0) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(kPairThreads, 1, 1);
+        cfg.dynamicSmemBytes = kPairSmem;
+        if (cudaOccupancyMaxActiveClusters(&n_pairs, attn_pair_kernel, &cfg) != cudaSuccess || n_pairs <= 0) {
+            (void)cudaGetLastError();
+            n_pairs = 74;
+        }
+        if (dev >= 0 && dev < 64) pairs_cached[dev] = n_pairs;
+    }
+    const int base = Hkv * a.n_layers * a.batch * p.n_row_groups;
+    const int max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens;
+    const size_t per_split = (size_t)Hkv * a.n_layers * a.batch * p.R_pad * (kD + 2) * sizeof(float);
+    // Split count by a small cost model (microseconds): whole waves of pairs, each pair paying a fixed set-up/drain cost
+    // plus its tiles; splitting adds the partial-result round trip through the workspace and the merge launch.
+    int best = 1;
+    double best_cost = 1e30;
+    const double t_tile = 0.8, t_cta = 6.0, t_partial = 3.0, t_merge_launch = 6.0;
+    const double avg_tiles = max_tiles + 1.0;  // context tiles + the tile of the step's own tokens
+    for (int s = 1; s <= 64; ++s) {
+        if (s > 1 && (s > max_tiles / 2 || per_split * s > a.partial_bytes)) break;  // at least two tiles per pair
+        const long long pairs = (long long)base * s;
+        const double waves = (double)((pairs + n_pairs - 1) / n_pairs);
+        double cost = waves * (t_cta + t_tile * (avg_tiles / s + (s > 1 ? 0.5 : 0.0)));
+        if (s > 1) cost += waves * t_partial + t_merge_launch + (double)per_split * s * 2.0 / 4.0e6;  // bytes / (4 TB/s) in us
+        if (cost < best_cost * 0.97) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    p.n_splits = best;
+    char* ws = reinterpret_cast<char*>(a.workspace) + a.partial_off;
+    p.part_o = reinterpret_cast<float*>(ws);
+    p.part_ml = reinterpret_cast<float*>(ws + (size_t)Hkv * a.n_layers * a.batch * p.n_splits * p.R_pad * kD * sizeof(float));
+
+    dim3 grid(2 * p.n_splits * p.n_row_groups, Hkv, a.n_layers * a.batch);
+    attn_pair_kernel<<<grid, kPairThreads, kPairSmem, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+    count_launch();
+    if (p.n_splits > 1) return launch_merge_tc(p, R_max, a.n_layers * a.batch, stream);
+    return SPECPV_OK;
+}
+
+}  // namespace specpv

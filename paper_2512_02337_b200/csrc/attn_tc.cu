@@ -17,86 +17,19 @@
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each, P_t aliases S_t.
 // With several KV splits the unnormalised (O, m, l) go to the workspace and merge_kernel combines
 // them by log-sum-exp.  Every wait is bounded; a wait that gives up records SPECPV_ERR_TIMEOUT.
-#include "tc_common.cuh"
+#include "attn_tc.cuh"
 
 namespace specpv {
 
 namespace {
 
 constexpr int kThreadsTc = 384;          // 12 warps
-constexpr int kTileTokens = 128;         // KV tokens per tile (128 / page size pages)
-constexpr int kD = 128;
 constexpr int kSlotBytes = 32768;        // one K or V tile: [2 d-halves][128 tokens][64 d] bf16
 constexpr int kStages = 5;
 constexpr int kQBytes = 2 * 32768;       // two row tiles
 constexpr int kSmemBytes = 1024 + kQBytes + kStages * kSlotBytes;
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
-constexpr float kSafeRowSum = 1.1529215e18f;  // 2^60: a tile's row sum below this cannot overflow the float32 sums
-
-struct TcParams {
-    CUtensorMap tm_q;      // (d, Hq, tokens)          box (64, G, 128/G)
-    CUtensorMap tm_knew;   // (d, Hkv, tokens)         box (64, 1, 64)
-    CUtensorMap tm_vnew;
-    CUtensorMap tm_kpool;  // (d, rows)                box (64, page size)
-    CUtensorMap tm_vpool;
-    const uint64_t* tree_mask;
-    const int32_t* q_lens;
-    const int32_t* block_table;
-    const int32_t* seq_lens;
-    void* out;
-    float* lse;
-    float* part_o;   // [lb][Hkv][splits][R_pad][128]
-    float* part_ml;  // [lb][Hkv][splits][R_pad][2]
-    void* workspace;
-    int layer0, batch, M_max, mask_words, Hq, Hkv, G, max_blocks, n_pages;
-    int n_splits, n_row_groups, R_pad, out_f32;
-    int bs;          // tokens per page (16, 32 or 64)
-    uint32_t pool_rows;  // rows of the pool tensor map (an out-of-range row coordinate reads zeros)
-    float scale_log2;
-};
 
 using namespace tc;
-
-// tcgen05.mma with the shared-memory descriptors given as (low word, common high word); `acc` = 0
-// overwrites D, anything else accumulates.
-__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                            uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
-        : "memory");
-}
-__device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                            uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
-        : "memory");
-}
-// keeps the compiler from hoisting per-instruction descriptor words out of the tile loop
-__device__ __forceinline__ uint32_t launder(uint32_t x) {
-    asm volatile("" : "+r"(x));
-    return x;
-}
-// acc.x += low bf16 of w, acc.y += high bf16 of w: the mixed-precision add takes the 16-bit halves as they
-// are, so the packed word needs no shift / mask to be widened first (the sums are the same bit for bit)
-__device__ __forceinline__ void add_bf16_pair(float2& acc, uint32_t w) {
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\t"
-        "add.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
-        : "+f"(acc.x), "+f"(acc.y)
-        : "r"(w));
-}
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
 
 // Instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128, N = 128.
 constexpr uint32_t kIdescQK = make_idesc(128, false);
@@ -627,13 +560,15 @@ bool attention_tc_supported(const AttnArgs& a) {
     return get_encode_fn() != nullptr;
 }
 
+specpv_status launch_merge_tc(const TcParams& p, int R_max, int n_lb, cudaStream_t stream) {
+    dim3 mgrid((R_max + kMergeRows - 1) / kMergeRows, p.Hkv, n_lb);
+    merge_tc_kernel<<<mgrid, 32 * kMergeRows, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
+    count_launch();
+    return SPECPV_OK;
+}
+
 specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return SPECPV_ERR_CUDA;
-        attr_set = true;
-    }
     TcParams p{};
     const int G = a.g.G, Hq = a.g.Hq, Hkv = a.g.Hkv;
     const uint64_t step_tokens = (uint64_t)a.n_layers * a.batch * a.M_max;
@@ -670,6 +605,9 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
     const int R_max = a.M_max * G;
     p.n_row_groups = (R_max + 255) / 256;
     p.R_pad = p.n_row_groups * 256;
+    if (attention_pair_wanted(a)) return launch_attention_pair(p, a, stream);
+
+    if (!set_smem_limit_once(reinterpret_cast<const void*>(attn_tc_kernel), kSmemBytes)) return SPECPV_ERR_CUDA;
     // KV splits: fill the 148 SMs (one CTA each) in whole waves as evenly as the workspace allows
     const int base = Hkv * a.n_layers * a.batch * p.n_row_groups;
     const int max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens;
@@ -701,12 +639,7 @@ specpv_status launch_attention_tc(const AttnArgs& a, cudaStream_t stream) {
     attn_tc_kernel<<<grid, kThreadsTc, kSmemBytes, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
-    if (p.n_splits > 1) {
-        dim3 mgrid((R_max + kMergeRows - 1) / kMergeRows, Hkv, a.n_layers * a.batch);
-        merge_tc_kernel<<<mgrid, 32 * kMergeRows, 0, stream>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
-        count_launch();
-    }
+    if (p.n_splits > 1) return launch_merge_tc(p, R_max, a.n_layers * a.batch, stream);
     return SPECPV_OK;
 }
 

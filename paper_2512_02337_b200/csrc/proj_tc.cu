@@ -311,12 +311,7 @@ bool proj_tc_supported(const ProjArgs& a) {
 }
 
 specpv_status launch_proj_tc(const ProjArgs& a, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProjSmem) != cudaSuccess)
-            return SPECPV_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!tc::set_smem_limit_once(reinterpret_cast<const void*>(proj_tc_kernel), kProjSmem)) return SPECPV_ERR_CUDA;
     if (a.tokens <= 0 || a.n_layers_call <= 0) return SPECPV_OK;
     ProjTcParams p{};
     p.n_pad = a.tokens >= kMaxTokTile ? kMaxTokTile : (a.tokens + 31) / 32 * 32;

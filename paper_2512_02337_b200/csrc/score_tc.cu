@@ -299,13 +299,9 @@ bool scores_tc_supported(int dtype, int d, int G, int M_max) {
 
 specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_layers_total, int max_nb,
                                cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(scores_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess ||
-            cudaFuncSetAttribute(scores_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess)
-            return SPECPV_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!tc::set_smem_limit_once(reinterpret_cast<const void*>(scores_tc_kernel<false>), kScoreSmem) ||
+        !tc::set_smem_limit_once(reinterpret_cast<const void*>(scores_tc_kernel<true>), kScoreSmem))
+        return SPECPV_ERR_CUDA;
     if (max_nb <= 0 || n_layers_call <= 0) return SPECPV_OK;
     ScoreTcParams p{};
     const uint64_t step_tokens = (uint64_t)n_layers_call * sp.batch * sp.M_max;
