@@ -8,14 +8,19 @@
 // pair-wide tcgen05.mma (cta_group::2, M = 256), issued by one thread of the even CTA, which read both CTAs'
 // shared memory, so a K/V byte is fetched from HBM once and read from shared memory once per pair.
 //
-// Work is organised in steps: step t loads K of tile t and V of tile t-3 into ring slot t % 5 and issues
-// PV(t-3) then QK(t).  S lives in one of THREE tensor-memory buffers (tile mod 3) and P(j) overwrites the first
-// half of S(j)'s own buffer, so that the softmax warps never wait for a buffer: the buffer of tile j is theirs from
-// the completion of QK(j) until they hand P(j) over, and QK(j+3), which reuses it, is issued behind PV(j) on the
-// in-order tensor pipe.  The only wait on the critical loop is the issuer's wait for P(j).
-//   warp 0      TMA producer (both CTAs): its Q tile per stretch, then per step its K and V halves through the block
-//               table (128-byte swizzle); completion is counted on the even CTA's barriers
-//   warp 1      MMA issuer (even CTA): per step  PV(t-3), QK(t), two commits (S ready; step done = slot free)
+// S lives in one of THREE tensor-memory buffers (tile mod 3) and P(j) overwrites the first half of S(j)'s own
+// buffer, so the softmax warps never wait for a buffer: the buffer of tile j is theirs from the completion of
+// QK(j) until they hand P(j) over; QK(j+3) reuses it once PV(j) has completed.
+// Issuing one tcgen05.mma costs its thread 55-60 cycles whatever the shape, against 64 cycles of execution for
+// 128x128x16 per SM, and the tensor pipe queues next to nothing ahead: one issuing thread that also waits and
+// commits cannot keep the pipe busy (measured: 84-98 cycles per instruction, 65 with two issuing warps).  So the
+// two streams have a warp each, ordered against one another by commit barriers only.
+//   warp 0      TMA producer (both CTAs): its Q tile per stretch, then per tile its halves of K (ring of 5) and of V
+//               (ring of 5, three tiles behind) through the block table (128-byte swizzle); completion is counted on
+//               the even CTA's barriers
+//   warp 1      PV issuer (even CTA): O += P(j) V_j once the 16 softmax warps have stored P(j); commit = V slot free,
+//               O holds PV(j)
+//   warp 3      QK issuer (even CTA): S(t) = Q K_t^T once PV(t-3) has completed; commits: S ready, K slot free
 //   warp 2      zeroes the rows of its V half past the valid tokens (ragged last tile, the step's own tokens)
 //   warps 4-11  softmax (both CTAs): a warp owns 16 rows, four threads per row (tcgen05.ld 16x256b), so the row
 //               maximum and the overflow check stay inside the warp; online softmax in the log2 domain with a
@@ -24,6 +29,8 @@
 // With several KV splits the unnormalised (O, m, l) go to the workspace and the merge kernel combines them by
 // log-sum-exp.  Every wait is bounded; a wait that gives up records SPECPV_ERR_TIMEOUT, stops its loop, raises
 // the abort flag of both CTAs, and the pair still drains its copies and frees its tensor memory.
+#include <limits.h>
+
 #include "attn_tc.cuh"
 
 namespace specpv {
@@ -33,11 +40,10 @@ namespace {
 using namespace tc;
 
 constexpr int kPairThreads = 384;   // 12 warps
-constexpr int kRing = 5;            // steps in flight per CTA
-constexpr int kSlot = 32768;        // [K half of tile t: 2 d-halves x 64 tokens x 64 d][V half of tile t-3: 128 tokens x 64 channels]
-constexpr int kVOff = 16384;
+constexpr int kRing = 5;            // K tiles and V tiles in flight per CTA (a ring each)
+constexpr int kHalf = 16384;        // a K slot [2 d-halves x 64 tokens x 64 d] or a V slot [128 tokens x 64 channels]
 constexpr int kQTile = 32768;       // [2 d-halves][128 rows][64 d]
-constexpr int kPairSmem = 1024 + 2 * kQTile + kRing * kSlot;
+constexpr int kPairSmem = 1024 + 2 * kQTile + 2 * kRing * kHalf;
 constexpr uint32_t kColO = 384;     // tensor-memory columns: S/P buffer b at b * 128, O behind them
 constexpr int kLag = 3;             // PV runs this many tiles behind QK (= number of S/P buffers)
 constexpr uint64_t kWaitNs = 2000000000ull;
@@ -52,8 +58,10 @@ constexpr uint32_t kIdescPV2 = idesc_pair(true);  // B (= V) is MN-major
 struct __align__(8) PairBars {
     uint64_t q_full[2];          // even CTA: both CTAs' Q tiles of a stretch have landed (transaction bytes)
     uint64_t q_empty[2];         // both: the last QK of the stretch that used this Q buffer has completed
-    uint64_t ld_full[kRing];     // even CTA: a step's K and V halves are in place (bytes + one "V ready" per CTA)
-    uint64_t step_done[kRing];   // both: the step's PV and QK have completed (its slot is free; O holds that PV)
+    uint64_t k_full[kRing];      // even CTA: both CTAs' halves of a K tile have landed
+    uint64_t k_empty[kRing];     // both: QK of the tile in this slot has completed
+    uint64_t v_full[kRing];      // even CTA: both halves of a V tile are in place (bytes + one "V ready" per CTA)
+    uint64_t v_empty[kRing];     // both: PV of the tile in this slot has completed (slot free, O holds that PV)
     uint64_t vfix_full[kRing];   // own: this CTA's V half of a tile that needs zeroed rows has landed
     uint64_t s_full[kLag];       // both: S(j) is complete
     uint64_t p_full[kLag];       // even CTA: all 16 softmax warps have stored P(j)
@@ -106,14 +114,35 @@ struct SegIter {
     }
 };
 
+// 2^x for a pair of finite x (clamped to [-126, 127]) on the FMA and integer pipes (the special-function unit, 16 exponentials per
+// cycle and SM, is the softmax's scarcest resource): x = n + f with n = round(x) taken from the low mantissa bits of
+// x + 1.5 * 2^23, f in [-0.5, 0.5], 2^f by a cubic with maximum relative error 7.5e-5 (the weight is rounded to
+// bfloat16, relative error 3.9e-3, right after), n added to the exponent field.
+__device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
+    const float kMagic = 12582912.f;  // 1.5 * 2^23
+    x.x = fminf(fmaxf(x.x, -126.f), 127.f);  // 2^127 and the like trip the caller's overflow check, as +inf would
+    x.y = fminf(fmaxf(x.y, -126.f), 127.f);
+    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 r = __ffma2_rn(make_float2(0.055171459913253784f, 0.055171459913253784f), f, make_float2(0.2426108568906784f, 0.2426108568906784f));
+    r = __ffma2_rn(r, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+    r = __ffma2_rn(r, f, make_float2(0.9999281167984009f, 0.9999281167984009f));
+    r.x = __int_as_float(__float_as_int(r.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(r.y) + (__float_as_int(t.y) << 23));
+    return r;
+}
+// which of the 16 column groups of a row pair take their exponentials on the FMA pipe (fast path only)
+constexpr uint32_t kFmaExpGroups = 0x1111u;  // groups 0, 4, 8, 12: a quarter (measured: 1577 cycles per tile with none, 1392 with 4, 1446 with 5)
+
 // Bounded wait for the pair kernel: a wait that gives up records the fault and raises the abort flag of both CTAs.
 __device__ __forceinline__ bool pair_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
                                                void* workspace, int where, uint64_t limit_ns) {
     const uint64_t t0 = global_ns();
     for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
         if (*abort_flag) return false;
-        if ((it & 255u) == 255u && global_ns() - t0 > limit_ns) {
+        if ((it & 15u) == 15u && global_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             st_cluster_u32(peer_abort, 1u);
             record_fault(workspace, SPECPV_ERR_TIMEOUT, where, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
@@ -157,7 +186,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
     }
 
     const uint32_t q_smem = smem_u32(smem);
-    const uint32_t kv_smem = q_smem + 2 * kQTile;
+    const uint32_t k_smem = q_smem + 2 * kQTile, v_smem = k_smem + kRing * kHalf;
     volatile int* abort_flag = &bars.abort_flag;
     const uint32_t peer_abort = mapa(smem_u32(&bars.abort_flag), rank ^ 1u);
 
@@ -172,8 +201,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
             mbar_init(smem_u32(&bars.p_full[i]), 16);  // one arrival per softmax warp of the pair
         }
         for (int s = 0; s < kRing; ++s) {
-            mbar_init(smem_u32(&bars.ld_full[s]), 3);  // the byte count's arrival + one "V half ready" per CTA
-            mbar_init(smem_u32(&bars.step_done[s]), 1);
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 3);  // the byte count's arrival + one "V half ready" per CTA
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
             mbar_init(smem_u32(&bars.vfix_full[s]), 1);
         }
         mbar_init(smem_u32(&bars.o_full), 1);
@@ -196,131 +227,180 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
 
     // barriers of the even CTA, as seen from this CTA
     const uint32_t lead_q_full0 = mapa(smem_u32(&bars.q_full[0]), 0);
-    const uint32_t lead_ld_full0 = mapa(smem_u32(&bars.ld_full[0]), 0);
+    const uint32_t lead_k_full0 = mapa(smem_u32(&bars.k_full[0]), 0);
+    const uint32_t lead_v_full0 = mapa(smem_u32(&bars.v_full[0]), 0);
     const uint32_t lead_p_full0 = mapa(smem_u32(&bars.p_full[0]), 0);
     const uint32_t lead_o_free = mapa(smem_u32(&bars.o_free), 0);
 
     // Register budget: the control warpgroup (warps 0-3) gives registers to the two softmax warpgroups.
+    // Block-table access of the two producer warps: the entry of the next tile is loaded while the current one is
+    // issued and only looked at when its tile comes up, so the load's latency never stalls the warp.
+    constexpr int kNoPage = INT_MIN;  // the block lies past the sequence: the copy engine fills zeros
+    const int ppt = kTileTokens / p.bs;  // pages per tile
+    auto page_load = [&](const Seg& s, int blk) {
+        return ((long long)blk * p.bs < s.seq_len && blk < p.max_blocks) ? __ldg(p.block_table + (size_t)s.b * p.max_blocks + blk) : kNoPage;
+    };
+    // pool row of a page (an out-of-range row makes the copy engine fill zeros); a bad entry is recorded and read as zeros
+    auto page_row = [&](const Seg& s, int blk, int page, bool report) {
+        if (page == kNoPage) return (int)p.pool_rows;
+        if (page < 0 || page >= p.n_pages) {
+            if (report) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, s.b, blk, page, s.l);
+            return (int)p.pool_rows;
+        }
+        return (((p.layer0 + s.l) * p.n_pages + page) * p.Hkv + s.h) * p.bs;  // < 2^31: checked on the host
+    };
+
+    // Register budget: the control warpgroup (warps 0-3) gives registers to the two softmax warpgroups.
     if (warp == 0) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        // =========================== TMA producer ================================================
-        // The whole warp runs the loop; lane 0 does the barrier bookkeeping, each copy is issued by its own lane.
-        // Step t brings K of tile t (stretch walker `k`) and V of tile t - 3 (walker `v`) into slot t % 5.
-        const int ppt = kTileTokens / p.bs;  // pages per tile
-        // K copies: lane 2 pg + half, pg < ppt / 2 (this CTA's 64 tokens), half = 64-channel half of d
-        // V copies: lane 16 + pg, pg < ppt (all 128 tokens, this CTA's 64 channels)
-        const bool k_lane = lane < ppt, v_lane = lane >= 16 && lane < 16 + ppt;
-        const int k_pg = lane >> 1, k_half = lane & 1, v_pg = lane - 16;
-        SegIter it_k, it_v;
-        Seg sk, sv;
-        bool have_k = it_k.next(p, sk), have_v = it_v.next(p, sv);
-        int jk = 0, jv = 0, sidx_k = 0;
+        // =========================== K producer (both CTAs) ======================================
+        // Per stretch its Q tile, then per tile this CTA's 64 tokens of K into the K ring.  The whole warp runs the
+        // loop; lane 0 does the barrier bookkeeping; lane 2 pg + half copies the 64-channel half `half` of page pg.
+        const bool k_lane = lane < ppt;
+        const int k_pg = lane >> 1, k_half = lane & 1;
+        SegIter it;
+        Seg s;
+        uint32_t t = 0;
         bool ok = true;
-        // pool row of this lane's page of context tile j of a stretch (an out-of-range row makes the copy engine fill zeros)
-        auto page_row = [&](const Seg& s, int j, bool is_k) {
-            int row = (int)p.pool_rows;
-            const int blk = (s.tile_begin + j) * ppt + (is_k ? (int)rank * (ppt >> 1) + k_pg : v_pg);
-            if ((long long)blk * p.bs < s.seq_len && blk < p.max_blocks) {
-                const int page = p.block_table[(size_t)s.b * p.max_blocks + blk];
-                if (page < 0 || page >= p.n_pages) {
-                    if (is_k ? k_half == 0 : rank == 0) record_fault(p.workspace, SPECPV_ERR_BAD_BLOCK_TABLE, s.b, blk, page, s.l);
-                } else {
-                    row = (int)((((long long)(p.layer0 + s.l) * p.n_pages + page) * p.Hkv + s.h) * p.bs);
-                }
-            }
-            return row;
-        };
-        for (uint32_t t = 0; ok && (have_k || have_v); ++t) {
-            if (have_k && jk == 0) {  // the stretch's Q tile, ahead of its first K tile
-                const int qb = sidx_k & 1;
-                if (sidx_k >= 2) ok = pair_wait(smem_u32(&bars.q_empty[qb]), ((sidx_k >> 1) - 1) & 1, abort_flag, peer_abort, p.workspace, 1);
-                if (!ok) break;
-                if (lane == 0) {
-                    if (rank == 0) mbar_expect_tx(smem_u32(&bars.q_full[qb]), 2 * kQTile);
-                    for (int half = 0; half < 2; ++half)
-                        tma_load_3d_pair(q_smem + qb * kQTile + half * 16384, &p.tm_q, half * 64, sk.h * p.G,
-                                         sk.lb * p.M_max + sk.tok0 + (int)rank * tok_per_tile, lead_q_full0 + qb * 8);
-                }
-                __syncwarp();
-            }
-            const uint32_t slot = t % kRing;
-            const bool do_v = have_v && t >= (uint32_t)kLag;
-            const bool fix = do_v && jv >= sv.first_fix;
-            int row_mine = (int)p.pool_rows;
-            if (k_lane && have_k && jk < sk.n_ctx) row_mine = page_row(sk, jk, true);
-            if (v_lane && do_v && jv < sv.n_ctx) row_mine = page_row(sv, jv, false);
-            if (t >= (uint32_t)kRing) ok = pair_wait(smem_u32(&bars.step_done[slot]), ((t / kRing) - 1) & 1, abort_flag, peer_abort, p.workspace, 2);
+        for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+            const int qb = sidx & 1;
+            if (sidx >= 2) ok = pair_wait(smem_u32(&bars.q_empty[qb]), ((sidx >> 1) - 1) & 1, abort_flag, peer_abort, p.workspace, 1);
             if (!ok) break;
-            const uint32_t slot_base = kv_smem + slot * kSlot;
-            const uint32_t full = lead_ld_full0 + slot * 8, vfix = smem_u32(&bars.vfix_full[slot]);
             if (lane == 0) {
-                if (rank == 0) mbar_expect_tx(smem_u32(&bars.ld_full[slot]), (have_k ? kSlot : 0) + ((do_v && !fix) ? kSlot : 0));
-                if (fix) mbar_expect_tx(vfix, kSlot - kVOff);
+                if (rank == 0) mbar_expect_tx(smem_u32(&bars.q_full[qb]), 2 * kQTile);
+                for (int half = 0; half < 2; ++half)
+                    tma_load_3d_pair(q_smem + qb * kQTile + half * 16384, &p.tm_q, half * 64, s.h * p.G,
+                                     s.lb * p.M_max + s.tok0 + (int)rank * tok_per_tile, lead_q_full0 + qb * 8);
             }
             __syncwarp();
-            if (have_k) {
-                if (jk >= sk.n_ctx) {  // the step's own tokens
-                    if (lane < 2)
-                        tma_load_3d_pair(slot_base + lane * 8192, &p.tm_knew, lane * 64, sk.h, sk.lb * p.M_max + (int)rank * 64, full);
+            int blk = s.tile_begin * ppt + (int)rank * (ppt >> 1) + k_pg;  // this lane's block of the current tile
+            int page_next = (k_lane && s.n_ctx > 0) ? page_load(s, blk) : kNoPage;
+            for (int j = 0; j < s.n_tiles; ++j, ++t, blk += ppt) {
+                const uint32_t ks = t % kRing;
+                const int page = page_next;
+                if (k_lane && j + 1 < s.n_ctx) page_next = page_load(s, blk + ppt);
+                if (t >= (uint32_t)kRing) ok = pair_wait(smem_u32(&bars.k_empty[ks]), ((t / kRing) - 1) & 1, abort_flag, peer_abort, p.workspace, 2);
+                if (!ok) break;
+                const uint32_t dst = k_smem + ks * kHalf, full = lead_k_full0 + ks * 8;
+                if (lane == 0 && rank == 0) mbar_expect_tx(smem_u32(&bars.k_full[ks]), 2 * kHalf);
+                __syncwarp();
+                if (j >= s.n_ctx) {  // the step's own tokens
+                    if (lane < 2) tma_load_3d_pair(dst + lane * 8192, &p.tm_knew, lane * 64, s.h, s.lb * p.M_max + (int)rank * 64, full);
                 } else if (k_lane) {
-                    tma_load_2d_pair(slot_base + k_half * 8192 + k_pg * p.bs * 128, &p.tm_kpool, k_half * 64, row_mine, full);
+                    tma_load_2d_pair(dst + k_half * 8192 + k_pg * p.bs * 128, &p.tm_kpool, k_half * 64, page_row(s, blk, page, k_half == 0), full);
                 }
             }
-            if (do_v) {
-                const uint32_t vbar = fix ? vfix : full;
-                if (jv >= sv.n_ctx) {
-                    if (lane == 16 || lane == 17)
-                        tma_load_3d_pair(slot_base + kVOff + (lane - 16) * 8192, &p.tm_vnew, (int)rank * 64, sv.h,
-                                         sv.lb * p.M_max + (lane - 16) * 64, vbar);
-                } else if (v_lane) {
-                    tma_load_2d_pair(slot_base + kVOff + v_pg * p.bs * 128, &p.tm_vpool, (int)rank * 64, row_mine, vbar);
-                }
-            }
-            __syncwarp();
-            if (lane == 0 && !fix) mbar_arrive_cluster(full);  // this CTA's V half needs no zeroing (or the step has none)
-            if (have_k && ++jk == sk.n_tiles) { have_k = it_k.next(p, sk); jk = 0; ++sidx_k; }
-            if (do_v && ++jv == sv.n_tiles) { have_v = it_v.next(p, sv); jv = 0; }
         }
     } else if (warp == 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        // =========================== MMA issuer (even CTA) =======================================
-        // One thread issues every contraction of the pair: per step  PV(t-3), QK(t).  PV(t-3) reads P from the
-        // buffer that QK(t) overwrites; the tensor pipe runs in order, so no wait lies between them.  The step and
-        // tile counters run across stretches, so the pipeline does not drain between them; only O is handed over.
+        // =========================== PV issuer (even CTA) ========================================
+        // O += P(j) V_j for every tile j, in order.  The whole warp runs the loop, lane 0 issues.  The tile counter
+        // runs across stretches; only O is handed over between them.
         if (rank == 0) {
             const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
-            const uint32_t q_lo0 = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
-            const uint32_t k_lo0 = ((kv_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
-            const uint32_t v_lo0 = (((kv_smem + kVOff) >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
-            SegIter it_k, it_v;  // it_k walks the QK side, it_v the PV side
-            Seg sk, sv;
-            bool have_k = it_k.next(p, sk), have_v = it_v.next(p, sv);
-            int jk = 0, jv = 0, sidx_k = 0, sidx_v = 0;
+            const uint32_t v_lo0 = ((v_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            SegIter it;
+            Seg s;
+            uint32_t g = 0;
             bool ok = true;
-            for (uint32_t t = 0; ok && (have_k || have_v); ++t) {
-                const uint32_t slot = t % kRing, buf = t % kLag;
-                const bool do_v = have_v && t >= (uint32_t)kLag;
-                if (have_k && jk == 0) ok = pair_wait(smem_u32(&bars.q_full[sidx_k & 1]), (sidx_k >> 1) & 1, abort_flag, peer_abort, p.workspace, 3);
-                if (ok) ok = pair_wait(smem_u32(&bars.ld_full[slot]), (t / kRing) & 1, abort_flag, peer_abort, p.workspace, 4);
-                if (ok && do_v) {
-                    if (jv == 0 && sidx_v > 0) ok = pair_wait(smem_u32(&bars.o_free), (sidx_v - 1) & 1, abort_flag, peer_abort, p.workspace, 6);
-                    if (ok) ok = pair_wait(smem_u32(&bars.p_full[buf]), ((t - kLag) / kLag) & 1, abort_flag, peer_abort, p.workspace, 7);
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after();
-                if (lane == 0) {
-                    if (do_v) {  // O += P(t-3) V
-                        const uint32_t b_lo = launder(v_lo0 + slot * (kSlot >> 4));
+            for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+                for (int j = 0; j < s.n_tiles; ++j, ++g) {
+                    const uint32_t vs = g % kRing, buf = g % kLag;
+                    ok = pair_wait(smem_u32(&bars.v_full[vs]), (g / kRing) & 1, abort_flag, peer_abort, p.workspace, 4);
+                    if (ok && j == 0 && sidx > 0) ok = pair_wait(smem_u32(&bars.o_free), (sidx - 1) & 1, abort_flag, peer_abort, p.workspace, 6);
+                    if (ok) ok = pair_wait(smem_u32(&bars.p_full[buf]), (g / kLag) & 1, abort_flag, peer_abort, p.workspace, 7);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t b_lo = launder(v_lo0 + vs * (kHalf >> 4));
                         const uint32_t a = tmem + buf * 128, d = tmem + kColO;
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk)  // 16 tokens per instruction: two 8-row groups of 1024 bytes
-                            mma2_ts_lohi(d, a + kk * 8, b_lo + (uint32_t)kk * (2048u >> 4), desc_hi, kIdescPV2, (jv > 0 || kk > 0) ? 1u : 0u);
-                        if (jv == sv.n_tiles - 1) tc_commit_pair(smem_u32(&bars.o_full));
+                            mma2_ts_lohi(d, a + kk * 8, b_lo + (uint32_t)kk * (2048u >> 4), desc_hi, kIdescPV2, (j > 0 || kk > 0) ? 1u : 0u);
+                        tc_commit_pair(smem_u32(&bars.v_empty[vs]));
+                        if (j == s.n_tiles - 1) tc_commit_pair(smem_u32(&bars.o_full));
                     }
-                    if (have_k) {  // S(t) = Q K^T
-                        const uint32_t a_lo = launder(q_lo0 + (uint32_t)(sidx_k & 1) * (kQTile >> 4));
-                        const uint32_t b_lo = launder(k_lo0 + slot * (kSlot >> 4));
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (warp == 2) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // =========================== V producer (both CTAs) ======================================
+        // Per tile this CTA's 64 channels of V (all 128 tokens) into the V ring; lane pg copies page pg.  Rows of a V tile
+        // past its valid tokens may hold anything (stale pages, rows of other sequences' steps): for a ragged last
+        // context tile and for the tile of the step's own tokens the copies complete on this CTA's own barrier, the
+        // warp zeroes those rows in its half (so that 0 * garbage cannot give NaN) and only then reports the half ready.
+        const bool v_lane = lane < ppt;
+        SegIter it;
+        Seg s;
+        uint32_t g = 0, fix_parity = 0;  // bit `slot`: parity of the next use of that slot's zeroing barrier
+        bool ok = true;
+        while (ok && it.next(p, s)) {
+            int blk = s.tile_begin * ppt + lane;
+            int page_next = (v_lane && s.n_ctx > 0) ? page_load(s, blk) : kNoPage;
+            for (int j = 0; j < s.n_tiles; ++j, ++g, blk += ppt) {
+                const uint32_t vs = g % kRing;
+                const int page = page_next;
+                if (v_lane && j + 1 < s.n_ctx) page_next = page_load(s, blk + ppt);
+                if (g >= (uint32_t)kRing) ok = pair_wait(smem_u32(&bars.v_empty[vs]), ((g / kRing) - 1) & 1, abort_flag, peer_abort, p.workspace, 16);
+                if (!ok) break;
+                const bool fix = j >= s.first_fix;
+                const uint32_t dst = v_smem + vs * kHalf, full = lead_v_full0 + vs * 8, vfix = smem_u32(&bars.vfix_full[vs]);
+                if (lane == 0) {
+                    if (fix) mbar_expect_tx(vfix, kHalf);
+                    if (rank == 0) {
+                        if (fix) mbar_arrive(smem_u32(&bars.v_full[vs]));  // the bytes are counted on the zeroing barriers
+                        else mbar_expect_tx(smem_u32(&bars.v_full[vs]), 2 * kHalf);
+                    }
+                }
+                __syncwarp();
+                const uint32_t vbar = fix ? vfix : full;
+                if (j >= s.n_ctx) {  // the step's own tokens
+                    if (lane < 2) tma_load_3d_pair(dst + lane * 8192, &p.tm_vnew, (int)rank * 64, s.h, s.lb * p.M_max + lane * 64, vbar);
+                } else if (v_lane) {
+                    tma_load_2d_pair(dst + lane * p.bs * 128, &p.tm_vpool, (int)rank * 64, page_row(s, blk, page, rank == 0), vbar);
+                }
+                __syncwarp();
+                if (fix) {
+                    ok = pair_wait(vfix, (fix_parity >> vs) & 1u, abort_flag, peer_abort, p.workspace, 8);
+                    if (!ok) break;
+                    fix_parity ^= 1u << vs;
+                    const int n_valid = max(j >= s.n_ctx ? s.M : min(kTileTokens, s.seq_len - (s.tile_begin + j) * kTileTokens), 0);
+                    uint8_t* v = smem + 2 * kQTile + (size_t)kRing * kHalf + (size_t)vs * kHalf;
+                    for (int i = lane; i < (kTileTokens - n_valid) * 8; i += 32)
+                        *reinterpret_cast<uint4*>(v + (size_t)(n_valid + (i >> 3)) * 128 + (i & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+                if (lane == 0) mbar_arrive_cluster(full);  // this CTA's V half is ready
+            }
+        }
+    } else if (warp == 3) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        // =========================== QK issuer (even CTA) ========================================
+        // S(t) = Q K_t^T into buffer t mod 3, which still holds P(t-3): not before PV(t-3) has completed (the two
+        // issuing warps are ordered by that commit barrier only).  QK runs up to three tiles ahead of the softmax.
+        if (rank == 0) {
+            const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
+            const uint32_t q_lo0 = ((q_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            const uint32_t k_lo0 = ((k_smem >> 4) & 0x3FFFu) | ((16u >> 4) << 16);
+            SegIter it;
+            Seg s;
+            uint32_t t = 0;
+            bool ok = true;
+            for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+                for (int j = 0; j < s.n_tiles; ++j, ++t) {
+                    const uint32_t ks = t % kRing, buf = t % kLag;
+                    if (j == 0) ok = pair_wait(smem_u32(&bars.q_full[sidx & 1]), (sidx >> 1) & 1, abort_flag, peer_abort, p.workspace, 3);
+                    if (ok) ok = pair_wait(smem_u32(&bars.k_full[ks]), (t / kRing) & 1, abort_flag, peer_abort, p.workspace, 13);
+                    if (ok && t >= (uint32_t)kLag)
+                        ok = pair_wait(smem_u32(&bars.v_empty[(t - kLag) % kRing]), ((t - kLag) / kRing) & 1, abort_flag, peer_abort, p.workspace, 14);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_lo = launder(q_lo0 + (uint32_t)(sidx & 1) * (kQTile >> 4));
+                        const uint32_t b_lo = launder(k_lo0 + ks * (kHalf >> 4));
                         const uint32_t d = tmem + buf * 128;
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {  // 16 channels of d per instruction
@@ -329,45 +409,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                             mma2_ss_lohi(d, a_lo + a_off, b_lo + b_off, desc_hi, kIdescQK2, kk > 0 ? 1u : 0u);
                         }
                         tc_commit_pair(smem_u32(&bars.s_full[buf]));
-                        if (jk == sk.n_tiles - 1) tc_commit_pair(smem_u32(&bars.q_empty[sidx_k & 1]));
+                        tc_commit_pair(smem_u32(&bars.k_empty[ks]));
+                        if (j == s.n_tiles - 1) tc_commit_pair(smem_u32(&bars.q_empty[sidx & 1]));
                     }
-                    tc_commit_pair(smem_u32(&bars.step_done[slot]));
+                    __syncwarp();
                 }
-                __syncwarp();
-                if (have_k && ++jk == sk.n_tiles) { have_k = it_k.next(p, sk); jk = 0; ++sidx_k; }
-                if (do_v && ++jv == sv.n_tiles) { have_v = it_v.next(p, sv); jv = 0; ++sidx_v; }
             }
         }
-    } else if (warp == 2) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-        // =========================== V fixer =====================================================
-        // Rows of a V tile past its valid tokens may hold anything (stale pages, rows of other sequences' steps): zero
-        // them in this CTA's half so that 0 * garbage cannot give NaN, then report the half ready.  Only a ragged last
-        // context tile and the tile of the step's own tokens need it; their V copies complete on this CTA's own barrier.
-        SegIter it;
-        Seg s;
-        uint32_t g = 0, fix_parity = 0;  // bit `slot`: parity of the next fix use of that slot's barrier
-        bool ok = true;
-        while (ok && it.next(p, s)) {
-            for (int j = s.first_fix; j < s.n_tiles; ++j) {
-                const uint32_t slot = (g + j + kLag) % kRing;  // V of tile g + j travels with step g + j + 3
-                ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.vfix_full[slot]), (fix_parity >> slot) & 1u, abort_flag,
-                                                       peer_abort, p.workspace, 8));
-                if (!ok) break;
-                fix_parity ^= 1u << slot;
-                const int n_valid = j >= s.n_ctx ? s.M : min(kTileTokens, s.seq_len - (s.tile_begin + j) * kTileTokens);
-                uint8_t* v = smem + 2 * kQTile + (size_t)slot * kSlot + kVOff;
-                const int n_rows = kTileTokens - max(n_valid, 0);
-                for (int i = lane; i < n_rows * 8; i += 32)
-                    *reinterpret_cast<uint4*>(v + (size_t)(max(n_valid, 0) + (i >> 3)) * 128 + (i & 7) * 16) = make_uint4(0, 0, 0, 0);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(lead_ld_full0 + slot * 8);
-            }
-            g += (uint32_t)s.n_tiles;
-        }
-    } else if (warp == 3) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // =========================== softmax / correction / epilogue ==============================
@@ -416,7 +464,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                 // P = 2^(s*scale - m) as bf16 pairs: word 2n + k/2 of P (row a or b, columns 8n + cq, + 1) goes to
                 // v[2n + k/2], whose own value was consumed earlier.  The row sums are taken over the ROUNDED weights
                 // the tensor core will use, so that O / l is an exact weighted average of V rows.
-                auto exp_rows = [&](float ma, float mb, float& sum_a, float& sum_b) {
+                auto exp_rows = [&](float ma, float mb, float& sum_a, float& sum_b, const uint32_t fma_groups) {
                     const float2 na = make_float2(-ma, -ma), nb = make_float2(-mb, -mb);
                     float2 acc_a[2], acc_b[2];
 #pragma unroll
@@ -425,8 +473,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                     for (int n = 0; n < 16; ++n) {
                         const float2 xa = __ffma2_rn(make_float2(__uint_as_float(v[4 * n]), __uint_as_float(v[4 * n + 1])), sc2, na);
                         const float2 xb = __ffma2_rn(make_float2(__uint_as_float(v[4 * n + 2]), __uint_as_float(v[4 * n + 3])), sc2, nb);
-                        const uint32_t wa = pack_bf16(ex2(xa.x), ex2(xa.y));
-                        const uint32_t wb = pack_bf16(ex2(xb.x), ex2(xb.y));
+                        uint32_t wa, wb;
+                        if ((fma_groups >> n) & 1u) {
+                            const float2 ea = exp2_fma_pair(xa), eb = exp2_fma_pair(xb);
+                            wa = pack_bf16(ea.x, ea.y);
+                            wb = pack_bf16(eb.x, eb.y);
+                        } else {
+                            wa = pack_bf16(ex2(xa.x), ex2(xa.y));
+                            wb = pack_bf16(ex2(xb.x), ex2(xb.y));
+                        }
                         v[2 * n] = wa;
                         v[2 * n + 1] = wb;
                         add_bf16_pair(acc_a[n & 1], wa);
@@ -443,7 +498,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                 float add_a = 0.f, add_b = 0.f;
                 bool general = j == 0 || masked;
                 if (!general) {
-                    exp_rows(m_a, m_b, add_a, add_b);
+                    exp_rows(m_a, m_b, add_a, add_b, kFmaExpGroups);
                     const bool bad = (valid_a && (!(add_a < kSafeRowSum) || m_a == -INFINITY)) ||
                                      (valid_b && (!(add_b < kSafeRowSum) || m_b == -INFINITY));
                     if (__any_sync(0xffffffffu, bad)) {
@@ -505,9 +560,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                     if (__any_sync(0xffffffffu, need_a || need_b)) {
                         const float fa = !need_a ? 1.f : (m_a == -INFINITY ? 0.f : ex2(m_a - mt_a));
                         const float fb = !need_b ? 1.f : (m_b == -INFINITY ? 0.f : ex2(m_b - mt_b));
-                        // O must hold PV(j-1) before it is rescaled: that is step j+2, whose commit frees its slot (the
-                        // barrier cannot run a phase ahead: that takes PV(j+4), which needs the P this warp has not stored)
-                        ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.step_done[(g + 2) % kRing]), ((g + 2) / kRing) & 1,
+                        // O must hold PV(j-1) before it is rescaled: the commit behind that PV frees its V slot (the barrier
+                        // cannot run a phase ahead: that takes PV(j+4), which needs the P this warp has not stored yet)
+                        ok = __all_sync(0xffffffffu, pair_wait(smem_u32(&bars.v_empty[(g - 1) % kRing]), ((g - 1) / kRing) & 1,
                                                                abort_flag, peer_abort, p.workspace, 10));
                         if (!ok) break;
                         tc_fence_after();
@@ -523,7 +578,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                         if (need_a) { l_a *= fa; m_a = mt_a; }
                         if (need_b) { l_b *= fb; m_b = mt_b; }
                     }
-                    exp_rows(m_a == -INFINITY ? 0.f : m_a, m_b == -INFINITY ? 0.f : m_b, add_a, add_b);
+                    exp_rows(m_a == -INFINITY ? 0.f : m_a, m_b == -INFINITY ? 0.f : m_b, add_a, add_b, 0u);
                 }
                 l_a += add_a;
                 l_b += add_b;
