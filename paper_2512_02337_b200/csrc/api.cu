@@ -80,7 +80,9 @@ WorkspacePlan plan_workspace(const Geometry& g, int n_layers_per_call, int max_b
     WorkspacePlan w{};
     const size_t base = (size_t)g.Hkv * n_layers_per_call * max_batch;
     const size_t R_pad = round_up((size_t)M_max * g.G, 256);
-    w.partial_off = kStatusBytes;
+    w.counter_off = kStatusBytes;
+    w.counter_bytes = kHeaderBytes - kStatusBytes;
+    w.partial_off = kHeaderBytes;
     // room for kMaxSplitCtas + base split results of R_pad rows of (d + 2) floats
     w.partial_bytes = round_up((kMaxSplitCtas + base) * R_pad * (g.d + 2) * sizeof(float), 256);
     w.staging_off = w.partial_off + w.partial_bytes;
@@ -122,6 +124,8 @@ static specpv_status verify_common(const specpv_config* cfg, int layer0, int n_l
     a.out = out; a.lse = lse; a.workspace = workspace;
     a.partial_off = w.partial_off;
     a.partial_bytes = workspace_bytes - w.partial_off < w.partial_bytes ? workspace_bytes - w.partial_off : w.partial_bytes;
+    a.counter_off = w.counter_off;
+    a.counter_bytes = w.counter_bytes;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (attention_tc_supported(a)) return launch_attention_tc(a, s);
     return launch_attention_simt(a, s);
@@ -361,7 +365,7 @@ SPECPV_EXPORT specpv_status specpv_verify_partial_static(const specpv_config* cf
     if (M_max > kMaxQTokens) return SPECPV_ERR_CAPACITY;
     if ((int64_t)partial->max_blocks * g.bs < (int64_t)g.budget_blocks * g.bs + g.buffer_tokens) return SPECPV_ERR_CAPACITY;
     // the fixed scratch must hold the partial results of at least two KV splits
-    const size_t scratch = (size_t)SPECPV_STATIC_SCRATCH_BYTES - kStatusBytes;
+    const size_t scratch = (size_t)SPECPV_STATIC_SCRATCH_BYTES - kHeaderBytes;
     const size_t per_split = (size_t)n_layers * partial->batch * g.Hkv * round_up((size_t)M_max * g.G, 256) *
                              (g.d + 2) * sizeof(float);
     if (per_split > scratch / 2) return SPECPV_ERR_CAPACITY;
@@ -381,7 +385,9 @@ SPECPV_EXPORT specpv_status specpv_verify_partial_static(const specpv_config* cf
     a.seq_lens = partial->seq_lens;
     a.max_blocks = partial->max_blocks; a.n_pages = partial->n_pages; a.max_seq_len = partial->max_seq_len;
     a.out = out; a.lse = lse; a.workspace = base;
-    a.partial_off = kStatusBytes;
+    a.counter_off = kStatusBytes;
+    a.counter_bytes = kHeaderBytes - kStatusBytes;
+    a.partial_off = kHeaderBytes;
     a.partial_bytes = scratch;
     st = attention_tc_supported(a) ? launch_attention_tc(a, s) : launch_attention_simt(a, s);
     if (st != SPECPV_OK) return st;
@@ -544,8 +550,9 @@ static specpv_status proj_dispatch(ProjArgs& a, const Geometry& g, int layer0, i
     a.layer0 = layer0; a.n_layers_call = n_layers; a.n_layers_total = g.n_layers;
     a.tokens = batch * M_max;
     a.workspace = workspace;
-    a.scratch_off = kStatusBytes;
-    a.scratch_bytes = workspace_bytes - kStatusBytes;
+    if (workspace_bytes < kHeaderBytes) return SPECPV_ERR_CAPACITY;
+    a.scratch_off = kHeaderBytes;
+    a.scratch_bytes = workspace_bytes - kHeaderBytes;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (proj_tc_supported(a)) return launch_proj_tc(a, s);
     return launch_proj_simt(a, s);

@@ -68,48 +68,86 @@ struct __align__(8) PairBars {
     uint64_t o_full;             // both: the last PV of a stretch has completed
     uint64_t o_free;             // even CTA: all 16 softmax warps have read O of the finished stretch
     uint64_t drain;              // even CTA: completion of whatever was issued before an abort
+    uint64_t rows_done;          // own: the eight softmax warps have written their rows of a shared unit / seen the ticket
     uint32_t tmem_base;
     int abort_flag;
+    int ticket;                  // own: this CTA's arrival number on a shared unit (read by its softmax warps)
 };
 
-// One stretch of KV tiles of one (layer, sequence, KV head, row group) processed by a pair.
+// One stretch of KV tiles of one unit = (layer, sequence, KV head, row group) processed by a pair.
 struct Seg {
-    int lb, b, l, h, rg, split;
+    int lb, b, l, h, rg;
     int M, seq_len, tok0;
-    int tile_begin;   // first context tile (128 tokens each) of the stretch
+    int tile_begin;   // first tile of the stretch within the unit (context tiles, then the tile of the step's own tokens)
     int n_ctx;        // context tiles in the stretch
     int n_tiles;      // n_ctx + 1 if the stretch ends with the tile of the step's own tokens
     int first_fix;    // first tile (stretch-local) whose V rows past the valid tokens must be zeroed; n_tiles if none
-    bool direct;      // the stretch covers the whole KV range: results are final
+    bool direct;      // the stretch covers the whole unit: results are final
+    int slot;         // otherwise: where its partial results go (two slots per pair)
+    int counter;      // ... the unit's arrival counter (one per CTA rank) ...
+    int p_first, n_seg;          // ... and the pairs that share the unit: p_first .. p_first + n_seg - 1
+    long long unit_x0;           // global index of the unit's first tile
 };
 
-// The stretches of a pair, in order.  Here: exactly one, given by the grid position.
+// The work of a launch is the sequence of all tiles of all units, unit after unit (layer-major, then sequence, KV
+// head, row group); a pair takes an equal contiguous share of that sequence, so it meets at most two units that it
+// shares with neighbouring pairs (their partial results are merged by whichever CTA finishes a shared unit last).
+// SegIter walks a pair's share unit by unit.  Lengths live on the device, so every role computes the split itself.
 struct SegIter {
-    bool done = false;
+    long long x = 0, x_end = 0, tiles_per_layer = 0, quota = 1;
+    bool first = true, ready = false;
+    __device__ static int row_groups(const TcParams& p, int M) { return (M * p.G + 255) / 256; }
+    __device__ static int seq_M(const TcParams& p, int b) {
+        const int M = p.q_lens ? p.q_lens[b] : p.M_max;
+        return min(max(M, 0), p.M_max);
+    }
+    __device__ void init(const TcParams& p) {
+        ready = true;
+        tiles_per_layer = 0;
+        for (int b = 0; b < p.batch; ++b) {
+            const int tiles = (max(p.seq_lens[b], 0) + kTileTokens - 1) / kTileTokens + 1;
+            tiles_per_layer += (long long)tiles * p.Hkv * row_groups(p, seq_M(p, b));
+        }
+        const long long total = tiles_per_layer * p.n_layers_call;
+        const long long n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+        quota = max((total + n_pairs - 1) / n_pairs, 1ll);
+        x = min(pair * quota, total);
+        x_end = min(x + quota, total);
+    }
     __device__ bool next(const TcParams& p, Seg& s) {
-        if (done) return false;
-        done = true;
-        const int pair_x = blockIdx.x >> 1;
-        s.split = pair_x % p.n_splits;
-        s.rg = pair_x / p.n_splits;
-        s.h = blockIdx.y;
-        s.lb = blockIdx.z;
-        s.b = s.lb % p.batch;
-        s.l = s.lb / p.batch;
-        s.seq_len = max(p.seq_lens[s.b], 0);
-        int M = p.q_lens ? p.q_lens[s.b] : p.M_max;
-        s.M = min(max(M, 0), p.M_max);
-        s.tok0 = s.rg * (256 / p.G);
-        const int total_tiles = (s.seq_len + kTileTokens - 1) / kTileTokens;
-        const int tiles_per_split = (total_tiles + p.n_splits - 1) / p.n_splits;
-        s.tile_begin = min(s.split * tiles_per_split, total_tiles);
-        const int tile_end = min(s.tile_begin + tiles_per_split, total_tiles);
-        const bool last_split = s.split == p.n_splits - 1;
-        s.n_ctx = tile_end - s.tile_begin;
-        s.n_tiles = s.n_ctx + (last_split ? 1 : 0);
-        const bool ragged_ctx = s.n_ctx > 0 && tile_end == total_tiles && (s.seq_len % kTileTokens) != 0;
-        s.first_fix = ragged_ctx ? s.n_ctx - 1 : ((last_split && s.M < kTileTokens) ? s.n_ctx : s.n_tiles);
-        s.direct = p.n_splits == 1;
+        if (!ready) init(p);
+        if (x >= x_end) return false;
+        s.l = (int)(x / tiles_per_layer);
+        long long r = x % tiles_per_layer;
+        int b = 0, tiles = 1, rgs = 1, M = 0, seq_len = 0;
+        for (;; ++b) {  // the sequence this tile belongs to
+            seq_len = max(p.seq_lens[b], 0);
+            M = seq_M(p, b);
+            tiles = (seq_len + kTileTokens - 1) / kTileTokens + 1;
+            rgs = row_groups(p, M);
+            const long long nb = (long long)tiles * p.Hkv * rgs;
+            if (r < nb || b == p.batch - 1) break;
+            r -= nb;
+        }
+        const int unit_in_b = (int)(r / tiles), off = (int)(r % tiles);
+        s.b = b; s.lb = s.l * p.batch + b; s.h = unit_in_b / rgs; s.rg = unit_in_b % rgs;
+        s.M = M; s.seq_len = seq_len; s.tok0 = s.rg * (256 / p.G);
+        const int n_ctx_unit = tiles - 1;
+        const int n = (int)min((long long)(tiles - off), x_end - x);
+        s.tile_begin = off;
+        s.n_tiles = n;
+        s.n_ctx = max(min(off + n, n_ctx_unit) - off, 0);
+        const bool ragged = (seq_len % kTileTokens) != 0;
+        const int fix_unit = ragged ? n_ctx_unit - 1 : (M < kTileTokens ? n_ctx_unit : tiles);  // unit-local
+        s.first_fix = min(max(fix_unit - off, 0), n);
+        s.direct = off == 0 && n == tiles;
+        s.slot = (int)(blockIdx.x >> 1) * 2 + (first ? 0 : 1);
+        s.unit_x0 = x - off;
+        s.p_first = (int)(s.unit_x0 / quota);
+        s.n_seg = (int)((s.unit_x0 + tiles - 1) / quota) - s.p_first + 1;
+        s.counter = ((s.lb * p.Hkv + s.h) * p.n_row_groups + s.rg) * 2;
+        first = false;
+        x += n;
         return true;
     }
 };
@@ -135,14 +173,69 @@ __device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
 // which of the 16 column groups of a row pair take their exponentials on the FMA pipe (fast path only)
 constexpr uint32_t kFmaExpGroups = 0x1111u;  // groups 0, 4, 8, 12: a quarter (measured: 1577 cycles per tile with none, 1392 with 4, 1446 with 5)
 
+// Log-sum-exp merge of the partial results of a unit shared between pairs, for the 128 rows of one CTA rank, by the
+// eight softmax warps of the CTA that finished the unit last (w8 = 0..7).  Warp w8 owns rows 16 w8 .. 16 w8 + 15; a
+// lane owns four channels of each of them, so a warp-wide load covers one whole row (512 contiguous bytes: with a
+// row half per thread instead, the same merge took 40 us for nine pairs).  Lane r < 16 keeps row r's running maximum
+// and sum.  Per pair all 16 row loads of a thread are in flight together; everything comes from L2.
+__device__ __forceinline__ void merge_shared_unit(const TcParams& p, const Seg& s, long long quota, int rank, int w8, int lane) {
+    const int row0 = rank * 128 + w8 * 16;  // first row (within the row group) of this warp
+    if (s.tok0 + row0 / p.G >= s.M) return;  // rows ascend with the token: none of this warp's rows is in use
+    float m_all = -INFINITY, l_all = 0.f;    // state of row row0 + lane (lanes 0..15)
+    float4 o[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) o[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < s.n_seg; ++q) {
+        const int slot = (s.p_first + q) * 2 + ((q == 0 && (long long)s.p_first * quota < s.unit_x0) ? 1 : 0);
+        const size_t prow0 = (size_t)slot * 256 + row0;
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (lane < 16) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml) + prow0 + lane);
+        const float4* src = reinterpret_cast<const float4*>(p.part_o + prow0 * kD) + lane;
+        float4 po[16];
+#pragma unroll
+        for (int r = 0; r < 16; ++r) po[r] = __ldcg(src + r * (kD / 4));
+        // this lane's row: new maximum, factor for what has been gathered so far, weight of this pair
+        const float m_new = fmaxf(m_all, ml.x);
+        const float f_mine = (m_all == -INFINITY || m_new == -INFINITY) ? 0.f : __expf(m_all - m_new);
+        const float w_mine = ml.x == -INFINITY ? 0.f : __expf(ml.x - m_new);
+        m_all = m_new;
+        l_all = fmaf(l_all, f_mine, ml.y * w_mine);
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+            const float f = __shfl_sync(0xffffffffu, f_mine, r), w = __shfl_sync(0xffffffffu, w_mine, r);
+            o[r].x = fmaf(o[r].x, f, po[r].x * w); o[r].y = fmaf(o[r].y, f, po[r].y * w);
+            o[r].z = fmaf(o[r].z, f, po[r].z * w); o[r].w = fmaf(o[r].w, f, po[r].w * w);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+        const int grow = row0 + r;
+        const int tok = s.tok0 + grow / p.G;
+        const float l_r = __shfl_sync(0xffffffffu, l_all, r), m_r = __shfl_sync(0xffffffffu, m_all, r);
+        if (tok >= s.M) continue;  // warp-uniform
+        const size_t out_row = ((size_t)s.lb * p.M_max + tok) * p.Hq + s.h * p.G + grow % p.G;
+        const float inv = 1.f / l_r;
+        const float4 v = make_float4(o[r].x * inv, o[r].y * inv, o[r].z * inv, o[r].w * inv);
+        if (p.out_f32) {
+            reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_row * kD)[lane] = v;
+        } else {
+            uint2 w2;
+            w2.x = pack_bf16(v.x, v.y);
+            w2.y = pack_bf16(v.z, v.w);
+            reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_row * kD)[lane] = w2;
+        }
+        if (p.lse && lane == 0) p.lse[out_row] = m_r + logf(l_r);
+    }
+}
+
 // Bounded wait for the pair kernel: a wait that gives up records the fault and raises the abort flag of both CTAs.
 __device__ __forceinline__ bool pair_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t peer_abort,
                                                void* workspace, int where, uint64_t limit_ns) {
     const uint64_t t0 = global_ns();
     for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((it & 15u) == 15u && global_ns() - t0 > limit_ns) {
+        if ((it & 255u) == 255u && global_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             st_cluster_u32(peer_abort, 1u);
             record_fault(workspace, SPECPV_ERR_TIMEOUT, where, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
@@ -167,22 +260,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
     const uint32_t rank = cluster_ctarank();  // 0: the CTA that issues the contractions and counts the completions
     const int tok_per_tile = 128 / p.G;       // step tokens per 128-row tile
 
-    // Uniform early exits (both CTAs of a pair see the same stretch).
+    // A pair without work leaves at once (uniform for both CTAs).
     {
         SegIter it;
-        Seg s;
-        it.next(p, s);
-        if (s.tok0 >= s.M) return;
-        if (s.n_tiles == 0) {
-            // an empty split: publish (m = -inf, l = 0) so that the merge ignores it
-            for (int r = threadIdx.x; r < 128; r += kPairThreads) {
-                const int row = s.rg * 256 + (int)rank * 128 + r;
-                const size_t prow = (((size_t)s.lb * p.Hkv + s.h) * p.n_splits + s.split) * p.R_pad + row;
-                p.part_ml[prow * 2] = -INFINITY;
-                p.part_ml[prow * 2 + 1] = 0.f;
-            }
-            return;
-        }
+        it.init(p);
+        if (it.x >= it.x_end) return;
     }
 
     const uint32_t q_smem = smem_u32(smem);
@@ -210,6 +292,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
         mbar_init(smem_u32(&bars.o_full), 1);
         mbar_init(smem_u32(&bars.o_free), 16);
         mbar_init(smem_u32(&bars.drain), 1);
+        mbar_init(smem_u32(&bars.rows_done), 8);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -429,7 +512,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         SegIter it;
         Seg s;
-        uint32_t g = 0;
+        uint32_t g = 0, rows_phase = 0;
         bool ok = true;
         for (int sidx = 0; ok && it.next(p, s); ++sidx) {
             const int row_a = (int)rank * 128 + ra, row_b = (int)rank * 128 + rb;  // rows within the row group
@@ -546,7 +629,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                     mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
                     mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
                     mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
-                    const float mt_a = mx_a * p.scale_log2, mt_b = mx_b * p.scale_log2;
+                    // The reference is a whole number of octaves (ceil(-inf) = -inf): weights 2^(x - m) taken against
+                    // references that differ by an integer differ by an exact power of two, so their bfloat16 roundings,
+                    // and with them the result, do not depend on where the KV range was cut between pairs.
+                    const float mt_a = ceilf(mx_a * p.scale_log2), mt_b = ceilf(mx_b * p.scale_log2);
                     // lazy rescale: keep the old reference unless the new maximum is more than 2^8 larger.  The decision
                     // is per row, the tensor-memory traffic is warp-wide (factor 1 where nothing changes).
                     bool need_a = false, need_b = false;
@@ -613,7 +699,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                 const int row = r ? row_b : row_a, tok = r ? tok_b : tok_a;
                 const float l_run = r ? l_b : l_a, m_run = r ? m_b : m_a;
                 const size_t out_row = ((size_t)s.lb * p.M_max + tok) * p.Hq + s.h * p.G + row % p.G;
-                const size_t prow = (((size_t)s.lb * p.Hkv + s.h) * p.n_splits + s.split) * p.R_pad + s.rg * 256 + row;
+                const size_t prow = (size_t)s.slot * 256 + row;
                 const float inv = s.direct ? 1.f / l_run : 1.f;
 #pragma unroll
                 for (int n = 0; n < 16; ++n) {
@@ -634,6 +720,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
                         p.part_ml[prow * 2] = m_run * kLn2;  // natural-log units for the merge
                         p.part_ml[prow * 2 + 1] = l_run;
                     }
+                }
+            }
+            if (!s.direct) {
+                // ---- a unit shared with other pairs: the CTA that arrives last (per CTA rank: each rank owns its 128
+                // rows) merges every pair's partial results by log-sum-exp.  Arrival counters live in the zeroed head of
+                // the workspace and are put back to zero by the merging CTA.
+                // (the eight warps meet on a shared-memory barrier with a bounded wait, not on bar.sync: after a wait that
+                // gave up somewhere a warp may never get here)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.rows_done));
+                if (warp == 4) {  // every warp of this CTA has written its rows: take a ticket
+                    ok = pair_wait(smem_u32(&bars.rows_done), rows_phase & 1, abort_flag, peer_abort, p.workspace, 17);
+                    if (ok && lane == 0) bars.ticket = atomicAdd(p.counters + s.counter + (int)rank, 1);
+                    __syncwarp();
+                } else {
+                    ok = pair_wait(smem_u32(&bars.rows_done), rows_phase & 1, abort_flag, peer_abort, p.workspace, 17);
+                }
+                if (!ok) break;
+                ++rows_phase;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.rows_done));  // second round: the ticket is in shared memory
+                ok = pair_wait(smem_u32(&bars.rows_done), rows_phase & 1, abort_flag, peer_abort, p.workspace, 18);
+                if (!ok) break;
+                ++rows_phase;
+                if (*reinterpret_cast<volatile int*>(&bars.ticket) == s.n_seg - 1) {
+                    __threadfence();
+                    merge_shared_unit(p, s, it.quota, (int)rank, warp - 4, lane);
+                    if (warp == 4 && lane == 0) p.counters[s.counter + (int)rank] = 0;
                 }
             }
         }
@@ -669,8 +784,7 @@ bool attention_pair_wanted(const AttnArgs& a) { return a.M_max * a.g.G > 128; }
 specpv_status launch_attention_pair(TcParams& p, const AttnArgs& a, cudaStream_t stream) {
     if (!set_smem_limit_once(reinterpret_cast<const void*>(attn_pair_kernel), kPairSmem)) return SPECPV_ERR_CUDA;
     const int Hkv = a.g.Hkv;
-    const int R_max = a.M_max * a.g.G;
-    // KV splits: fill the pairs the device can hold at once (one CTA per SM) in whole waves
+    // one pair per two SMs the device can hold at once; a persistent grid, the work split evenly inside the kernel
     static int pairs_cached[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return SPECPV_ERR_CUDA;
@@ -686,36 +800,26 @@ specpv_status launch_attention_pair(TcParams& p, const AttnArgs& a, cudaStream_t
         }
         if (dev >= 0 && dev < 64) pairs_cached[dev] = n_pairs;
     }
-    const int base = Hkv * a.n_layers * a.batch * p.n_row_groups;
-    const int max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens;
-    const size_t per_split = (size_t)Hkv * a.n_layers * a.batch * p.R_pad * (kD + 2) * sizeof(float);
-    // Split count by a small cost model (microseconds): whole waves of pairs, each pair paying a fixed set-up/drain cost
-    // plus its tiles; splitting adds the partial-result round trip through the workspace and the merge launch.
-    int best = 1;
-    double best_cost = 1e30;
-    const double t_tile = 0.8, t_cta = 6.0, t_partial = 3.0, t_merge_launch = 6.0;
-    const double avg_tiles = max_tiles + 1.0;  // context tiles + the tile of the step's own tokens
-    for (int s = 1; s <= 64; ++s) {
-        if (s > 1 && (s > max_tiles / 2 || per_split * s > a.partial_bytes)) break;  // at least two tiles per pair
-        const long long pairs = (long long)base * s;
-        const double waves = (double)((pairs + n_pairs - 1) / n_pairs);
-        double cost = waves * (t_cta + t_tile * (avg_tiles / s + (s > 1 ? 0.5 : 0.0)));
-        if (s > 1) cost += waves * t_partial + t_merge_launch + (double)per_split * s * 2.0 / 4.0e6;  // bytes / (4 TB/s) in us
-        if (cost < best_cost * 0.97) {
-            best_cost = cost;
-            best = s;
-        }
-    }
-    p.n_splits = best;
+    const long long units = (long long)Hkv * a.n_layers * a.batch * p.n_row_groups;
+    const long long max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens + 1;  // context tiles + the step's own tokens
+    // no more pairs than give each at least two tiles (a pair's set-up costs about as much as four)
+    long long use = units * max_tiles / 2;
+    if (use < 1) use = 1;
+    if (use > n_pairs) use = n_pairs;
+    // partial results: two slots of 256 rows per pair; arrival counters: two per unit
+    const size_t slot_bytes = (size_t)256 * (kD + 2) * sizeof(float);
+    if ((size_t)use * 2 * slot_bytes > a.partial_bytes) use = (long long)(a.partial_bytes / (2 * slot_bytes));  // fewer pairs: slower, same result
+    if (use < 1 || (size_t)units * 2 * sizeof(int32_t) > a.counter_bytes) return SPECPV_ERR_CAPACITY;
     char* ws = reinterpret_cast<char*>(a.workspace) + a.partial_off;
     p.part_o = reinterpret_cast<float*>(ws);
-    p.part_ml = reinterpret_cast<float*>(ws + (size_t)Hkv * a.n_layers * a.batch * p.n_splits * p.R_pad * kD * sizeof(float));
+    p.part_ml = reinterpret_cast<float*>(ws + (size_t)use * 2 * 256 * kD * sizeof(float));
+    p.counters = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(a.workspace) + a.counter_off);
+    p.n_layers_call = a.n_layers;
+    p.n_splits = 1;
 
-    dim3 grid(2 * p.n_splits * p.n_row_groups, Hkv, a.n_layers * a.batch);
-    attn_pair_kernel<<<grid, kPairThreads, kPairSmem, stream>>>(p);
+    attn_pair_kernel<<<dim3((unsigned)(2 * use), 1, 1), kPairThreads, kPairSmem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return SPECPV_ERR_CUDA;
     count_launch();
-    if (p.n_splits > 1) return launch_merge_tc(p, R_max, a.n_layers * a.batch, stream);
     return SPECPV_OK;
 }
 

@@ -24,9 +24,11 @@ struct TcParams {
     const int32_t* seq_lens;
     void* out;
     float* lse;
-    float* part_o;   // [lb][Hkv][splits][R_pad][128]
-    float* part_ml;  // [lb][Hkv][splits][R_pad][2]
+    float* part_o;   // [lb][Hkv][splits][R_pad][128]  (pair kernel: [pair][2][256][128])
+    float* part_ml;  // [lb][Hkv][splits][R_pad][2]    (pair kernel: [pair][2][256][2])
+    int32_t* counters;  // pair kernel: arrival counters of shared units, [unit][CTA rank], zero between launches
     void* workspace;
+    int n_layers_call;
     int layer0, batch, M_max, mask_words, Hq, Hkv, G, max_blocks, n_pages;
     int n_splits, n_row_groups, R_pad, out_f32;
     int bs;          // tokens per page (16, 32 or 64)

@@ -28,6 +28,9 @@ __device__ __forceinline__ void record_fault(void* workspace, int code, int i0, 
 }
 
 constexpr size_t kStatusBytes = 256;
+// Head of every workspace: the status word, then arrival counters of KV ranges shared between CTAs (two per (layer,
+// sequence, KV head, group of 256 rows) of a call; zero between launches).  All scratch starts behind it.
+constexpr size_t kHeaderBytes = 256 * 1024;
 constexpr int kMaxQTokens = 128;      // M_max supported by the attention kernels (two mask words)
 constexpr int kMaxSplitCtas = 8 * 148;  // the workspace holds split-KV partial results of this many CTAs (+ one per head)
 
@@ -50,6 +53,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- workspace carving --------------------------------------------------------------------
 struct WorkspacePlan {
+    size_t counter_off, counter_bytes;  // arrival counters of KV ranges shared between CTAs (zero between launches)
     size_t partial_off, partial_bytes;  // split-KV partial results
     size_t staging_off, staging_bytes;  // device copies of host step tensors (specpv_verify_host)
     size_t total;
@@ -88,6 +92,7 @@ struct AttnArgs {
     float* lse;
     void* workspace;
     size_t partial_off, partial_bytes;
+    size_t counter_off, counter_bytes;
 };
 
 specpv_status launch_attention_simt(const AttnArgs& a, cudaStream_t stream);

@@ -83,6 +83,8 @@ SPECPV_EXPORT specpv_status specpv_verify_full_offloaded(const specpv_config* cf
         a.workspace = workspace;
         a.partial_off = w.partial_off;
         a.partial_bytes = workspace_bytes - w.partial_off < w.partial_bytes ? workspace_bytes - w.partial_off : w.partial_bytes;
+        a.counter_off = w.counter_off;
+        a.counter_bytes = w.counter_bytes;
         st = attention_tc_supported(a) ? launch_attention_tc(a, s) : launch_attention_simt(a, s);
         ok = cudaEventRecord(done[slot], s) == cudaSuccess;
     }
