@@ -31,6 +31,8 @@
  *   Knew, Vnew    [n_layers_in_call][batch][M_max][Hkv][d]   keys/values of the step's own tokens
  *   tree_mask     [batch][M_max][W] uint64, W = ceil(M_max/64); bit a of row j: token j sees token a
  *   q_lens        [batch] int32   rows actually used per sequence (<= M_max); NULL = M_max for all
+ *                 M_max (chain + tree of a step) is at most 128: a larger value makes the verify calls
+ *                 return SPECPV_ERR_CAPACITY
  *   LSE           [n_layers_in_call][batch][M_max][Hq] float32 (natural log)
  *   summaries     kmax, kmin [n_layers][batch][Hkv][max_blocks][d]   (indexed by LOGICAL block)
  *   scores        [n_layers_in_call][batch][Hkv][max_blocks] float32
@@ -103,9 +105,12 @@ typedef struct {
 /* Human-readable name of a status code (static string, never NULL). */
 const char *specpv_status_string(specpv_status s);
 
-/* Bytes of device workspace that any call below needs for the given limits.  The first 256 bytes
- * hold the device status word and must be zeroed once by the caller (cudaMemset) before first use;
- * the rest is scratch (split-KV partial results, host-call staging) with no state between calls. */
+/* Bytes of device workspace that any call below needs for the given limits.  The first
+ * SPECPV_WORKSPACE_HEAD_BYTES hold the device status word and the arrival counters of KV ranges that
+ * several CTAs share; the caller zeroes them once (cudaMemset) before first use and the library
+ * leaves them zero after every call that completes (after SPECPV_ERR_TIMEOUT zero them again).  The
+ * rest is scratch (split-KV partial results, host-call staging) with no state between calls. */
+#define SPECPV_WORKSPACE_HEAD_BYTES (256u << 10)
 size_t specpv_workspace_bytes(const specpv_config *cfg, int n_layers_per_call, int max_batch,
                               int max_seq_len, int M_max);
 
@@ -171,7 +176,12 @@ specpv_status specpv_refresh_partial(const specpv_config *cfg, const specpv_page
 /* Section 3.2 / Algorithm 1 "TreeDecode" with KV_in = KV_partial: tree-masked GQA attention of
  * the step's tokens over the partial segment (sink | retrieval | local | buffer) followed by the
  * step's own keys under the tree mask.  out (and lse if not NULL) are fully written for rows
- * < q_lens[b]. */
+ * < q_lens[b].
+ * Two tensor-core kernels serve bfloat16 / head_dim 128: by default one CTA per KV range; with the
+ * environment variable SPECPV_ATTN_KERNEL=pair (read at every call) shapes with more than 128 query
+ * rows per KV head (M_max * Hq / Hkv) run on a kernel that gives a pair of SMs the two halves of
+ * those rows.  The results agree within the tolerance of either; the default is the faster one when
+ * steps follow one another (see the comment at attention_pair_wanted). */
 specpv_status specpv_verify_partial(const specpv_config *cfg, int layer0, int n_layers, const void *q,
                                     const void *k_new, const void *v_new, const uint64_t *tree_mask,
                                     const int32_t *q_lens, int M_max, const specpv_paged_kv *partial,
@@ -202,7 +212,8 @@ specpv_status specpv_verify_full(const specpv_config *cfg, int layer0, int n_lay
  * specpv_verify_partial.
  *
  * Limit: n_layers * batch * Hkv * ceil(M_max * G / 256) * 256 * (head_dim + 2) * 4 bytes (one
- * KV split's partial results) must fit twice into SPECPV_STATIC_SCRATCH_BYTES - 256; a larger
+ * KV split's partial results) must fit twice into SPECPV_STATIC_SCRATCH_BYTES -
+ * SPECPV_WORKSPACE_HEAD_BYTES; a larger
  * request returns SPECPV_ERR_CAPACITY and launches nothing.  Within the limit the scratch only
  * bounds how many KV splits are used, never the result.
  *
@@ -210,8 +221,9 @@ specpv_status specpv_verify_full(const specpv_config *cfg, int layer0, int n_lay
  * make that first call outside any stream capture.  Every call uses the same array: two calls
  * whose kernels can overlap on the GPU (different streams without an ordering between them) race
  * on it; calls on one stream, or ordered by events, are safe.  The array keeps the previous
- * call's partial results; nothing in it needs to start at zero except the status word, which the
- * call clears on `stream` before launching.  device_status (device, 5 x int32, nullable) receives
+ * call's partial results; its head (status word, arrival counters) starts at zero because the array
+ * is zero-initialised with the library image, the counters are back at zero when a call completes,
+ * and the status word is cleared on `stream` before launching.  device_status (device, 5 x int32, nullable) receives
  * a copy of the status word at the end of the call's work on `stream`: word 0 is the first
  * device-detected specpv_status of this call (0 = none), words 1..4 its details. */
 #define SPECPV_STATIC_SCRATCH_BYTES (16u << 20)
@@ -237,6 +249,10 @@ specpv_status specpv_verify_host(const specpv_config *cfg, int mode, int layer0,
 /* Section 3.2 (buffer) / Section 3.3 (removing invalid tokens): append rows accepted[b][0..n) of
  * Knew/Vnew (device int32 [batch][A_max], n = n_accepted[b] device [batch]) to cache `dst` at token
  * positions seq_lens[b].., then seq_lens[b] += n (seq_lens is dst->seq_lens, written in place).
+ * Layers may be committed in groups (layer0, n_layers), in ascending order: every group writes its
+ * rows at the lengths as they stand, and the lengths advance with the group that contains the
+ * model's last layer (layer0 + n_layers == cfg->n_layers), so a step's commit must end with that
+ * group and include every layer exactly once.
  * Rejected candidates are simply never appended.  If kmax/kmin are not NULL the summaries of the
  * touched blocks are recomputed.  A sequence whose cache would overflow is skipped and
  * SPECPV_ERR_CAPACITY recorded in the status word. */

@@ -138,14 +138,9 @@ def select(scores, sink_blocks: int, local_blocks: int, budget_blocks: int) -> n
 def head_shared_scores(scores) -> np.ndarray:
     """Scores that head-shared selection ranks on: the mean over the KV heads of one layer and sequence.
 
-    scores [Hkv][nb] float32 -> [nb] float32.  A ranking decision is taken in the precision of the path under
-    test, so the mean is formed in float32, head by head in order, then scaled by the float32 reciprocal of the
-    head count; the selection itself is :func:`select` on the result."""
-    s = np.asarray(scores, dtype=np.float32)
-    acc = np.zeros(s.shape[1], dtype=np.float32)
-    for h in range(s.shape[0]):
-        acc = (acc + s[h]).astype(np.float32)
-    return (acc * np.float32(np.float32(1.0) / np.float32(s.shape[0]))).astype(np.float32)
+    scores [Hkv][nb] -> [nb] float64: the plain mean, in double precision; the selection itself is :func:`select`
+    on the result."""
+    return np.asarray(scores, dtype=np.float64).mean(axis=0)
 
 
 def gather(k_pool, v_pool, block_table, seq_len: int, idx, pk_pool, pv_pool, first_page: int) -> int:

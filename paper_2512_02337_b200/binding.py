@@ -211,6 +211,7 @@ def specpv_verify_partial(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_l
 
 
 STATIC_SCRATCH_BYTES = 16 << 20
+WORKSPACE_HEAD_BYTES = 256 << 10  # SPECPV_WORKSPACE_HEAD_BYTES: status word and arrival counters, zero between calls
 
 
 def specpv_verify_partial_static(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, partial: Cache,

@@ -30,6 +30,8 @@
 // log-sum-exp.  Every wait is bounded; a wait that gives up records SPECPV_ERR_TIMEOUT, stops its loop, raises
 // the abort flag of both CTAs, and the pair still drains its copies and frees its tensor memory.
 #include <limits.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "attn_tc.cuh"
 
@@ -103,6 +105,10 @@ struct SegIter {
     }
     __device__ void init(const TcParams& p) {
         ready = true;
+        if (p.pairs_per_unit > 0) {  // the one stretch of this pair is worked out in next()
+            x = 0; x_end = 1; quota = 1;
+            return;
+        }
         tiles_per_layer = 0;
         for (int b = 0; b < p.batch; ++b) {
             const int tiles = (max(p.seq_lens[b], 0) + kTileTokens - 1) / kTileTokens + 1;
@@ -117,6 +123,37 @@ struct SegIter {
     __device__ bool next(const TcParams& p, Seg& s) {
         if (!ready) init(p);
         if (x >= x_end) return false;
+        if (p.pairs_per_unit > 0) {
+            // With fewer units than pairs every unit gets k pairs of its own, each an equal part of the unit's tiles: no
+            // pair meets two units (which would cost it a second Q tile, first tile and epilogue).
+            x = x_end;
+            const int k = p.pairs_per_unit, pair = (int)(blockIdx.x >> 1), unit = pair / k, part = pair % k;
+            s.rg = unit % p.n_row_groups;
+            s.h = (unit / p.n_row_groups) % p.Hkv;
+            s.lb = unit / (p.n_row_groups * p.Hkv);
+            s.b = s.lb % p.batch; s.l = s.lb / p.batch;
+            s.seq_len = max(p.seq_lens[s.b], 0);
+            s.M = seq_M(p, s.b);
+            s.tok0 = s.rg * (256 / p.G);
+            if (s.tok0 >= s.M) return false;  // no step tokens in this row group
+            const int n_ctx_unit = (s.seq_len + kTileTokens - 1) / kTileTokens, tiles = n_ctx_unit + 1;
+            const int per = (tiles + k - 1) / k, off = part * per;
+            if (off >= tiles) return false;
+            const int n = min(per, tiles - off);
+            s.tile_begin = off;
+            s.n_tiles = n;
+            s.n_ctx = max(min(off + n, n_ctx_unit) - off, 0);
+            const bool ragged = (s.seq_len % kTileTokens) != 0;
+            const int fix_unit = ragged ? n_ctx_unit - 1 : (s.M < kTileTokens ? n_ctx_unit : tiles);
+            s.first_fix = min(max(fix_unit - off, 0), n);
+            s.n_seg = (tiles + per - 1) / per;
+            s.direct = s.n_seg == 1;
+            s.slot = pair * 2;
+            s.p_first = unit * k;
+            s.unit_x0 = s.p_first;  // with quota = 1: every partial result sits in its pair's first slot
+            s.counter = unit * 2;
+            return true;
+        }
         s.l = (int)(x / tiles_per_layer);
         long long r = x % tiles_per_layer;
         int b = 0, tiles = 1, rgs = 1, M = 0, seq_len = 0;
@@ -174,57 +211,67 @@ __device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
 constexpr uint32_t kFmaExpGroups = 0x1111u;  // groups 0, 4, 8, 12: a quarter (measured: 1577 cycles per tile with none, 1392 with 4, 1446 with 5)
 
 // Log-sum-exp merge of the partial results of a unit shared between pairs, for the 128 rows of one CTA rank, by the
-// eight softmax warps of the CTA that finished the unit last (w8 = 0..7).  Warp w8 owns rows 16 w8 .. 16 w8 + 15; a
-// lane owns four channels of each of them, so a warp-wide load covers one whole row (512 contiguous bytes: with a
-// row half per thread instead, the same merge took 40 us for nine pairs).  Lane r < 16 keeps row r's running maximum
-// and sum.  Per pair all 16 row loads of a thread are in flight together; everything comes from L2.
+// eight softmax warps of the CTA that finished the unit last (w8 = 0..7).  Warp w8 owns rows 16 w8 .. 16 w8 + 15, in two
+// passes of eight; a lane owns four channels of each, so a warp-wide load covers one whole row (512 contiguous bytes:
+// with a row half per thread instead, the same merge took 40 us for nine pairs).  Everything comes from L2 at 1.5-2 us
+// per dependent round trip, so the partial rows of four pairs x eight rows are requested together.  Lane r < 8 keeps
+// row r's running maximum and sum.
 __device__ __forceinline__ void merge_shared_unit(const TcParams& p, const Seg& s, long long quota, int rank, int w8, int lane) {
-    const int row0 = rank * 128 + w8 * 16;  // first row (within the row group) of this warp
-    if (s.tok0 + row0 / p.G >= s.M) return;  // rows ascend with the token: none of this warp's rows is in use
-    float m_all = -INFINITY, l_all = 0.f;    // state of row row0 + lane (lanes 0..15)
-    float4 o[16];
+    auto slot_of = [&](int q) { return (s.p_first + q) * 2 + ((q == 0 && (long long)s.p_first * quota < s.unit_x0) ? 1 : 0); };
+    for (int pass = 0; pass < 2; ++pass) {
+        const int row0 = rank * 128 + w8 * 16 + pass * 8;  // first row (within the row group) of this pass
+        if (s.tok0 + row0 / p.G >= s.M) return;              // rows ascend with the token: no row in use from here on
+        float m_all = -INFINITY, l_all = 0.f;                // state of row row0 + lane (lanes 0..7)
+        float4 o[8];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) o[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int q = 0; q < s.n_seg; ++q) {
-        const int slot = (s.p_first + q) * 2 + ((q == 0 && (long long)s.p_first * quota < s.unit_x0) ? 1 : 0);
-        const size_t prow0 = (size_t)slot * 256 + row0;
-        float2 ml = make_float2(-INFINITY, 0.f);
-        if (lane < 16) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml) + prow0 + lane);
-        const float4* src = reinterpret_cast<const float4*>(p.part_o + prow0 * kD) + lane;
-        float4 po[16];
+        for (int r = 0; r < 8; ++r) o[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int q0 = 0; q0 < s.n_seg; q0 += 4) {
+            float2 ml[4];
+            float4 po[4][8];
 #pragma unroll
-        for (int r = 0; r < 16; ++r) po[r] = __ldcg(src + r * (kD / 4));
-        // this lane's row: new maximum, factor for what has been gathered so far, weight of this pair
-        const float m_new = fmaxf(m_all, ml.x);
-        const float f_mine = (m_all == -INFINITY || m_new == -INFINITY) ? 0.f : __expf(m_all - m_new);
-        const float w_mine = ml.x == -INFINITY ? 0.f : __expf(ml.x - m_new);
-        m_all = m_new;
-        l_all = fmaf(l_all, f_mine, ml.y * w_mine);
+            for (int u = 0; u < 4; ++u) {
+                const size_t prow0 = (size_t)slot_of(min(q0 + u, s.n_seg - 1)) * 256 + row0;
+                ml[u] = make_float2(-INFINITY, 0.f);
+                if (lane < 8 && q0 + u < s.n_seg) ml[u] = __ldcg(reinterpret_cast<const float2*>(p.part_ml) + prow0 + lane);
+                const float4* src = reinterpret_cast<const float4*>(p.part_o + prow0 * kD) + lane;
 #pragma unroll
-        for (int r = 0; r < 16; ++r) {
-            const float f = __shfl_sync(0xffffffffu, f_mine, r), w = __shfl_sync(0xffffffffu, w_mine, r);
-            o[r].x = fmaf(o[r].x, f, po[r].x * w); o[r].y = fmaf(o[r].y, f, po[r].y * w);
-            o[r].z = fmaf(o[r].z, f, po[r].z * w); o[r].w = fmaf(o[r].w, f, po[r].w * w);
+                for (int r = 0; r < 8; ++r) po[u][r] = __ldcg(src + r * (kD / 4));
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                // this lane's row: new maximum, factor for what has been gathered so far, weight of this pair
+                const float m_new = fmaxf(m_all, ml[u].x);
+                const float f_mine = (m_all == -INFINITY || m_new == -INFINITY) ? 0.f : __expf(m_all - m_new);
+                const float w_mine = ml[u].x == -INFINITY ? 0.f : __expf(ml[u].x - m_new);
+                m_all = m_new;
+                l_all = fmaf(l_all, f_mine, ml[u].y * w_mine);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const float f = __shfl_sync(0xffffffffu, f_mine, r), w = __shfl_sync(0xffffffffu, w_mine, r);
+                    o[r].x = fmaf(o[r].x, f, w == 0.f ? 0.f : po[u][r].x * w); o[r].y = fmaf(o[r].y, f, w == 0.f ? 0.f : po[u][r].y * w);
+                    o[r].z = fmaf(o[r].z, f, w == 0.f ? 0.f : po[u][r].z * w); o[r].w = fmaf(o[r].w, f, w == 0.f ? 0.f : po[u][r].w * w);
+                }
+            }
         }
-    }
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        const int grow = row0 + r;
-        const int tok = s.tok0 + grow / p.G;
-        const float l_r = __shfl_sync(0xffffffffu, l_all, r), m_r = __shfl_sync(0xffffffffu, m_all, r);
-        if (tok >= s.M) continue;  // warp-uniform
-        const size_t out_row = ((size_t)s.lb * p.M_max + tok) * p.Hq + s.h * p.G + grow % p.G;
-        const float inv = 1.f / l_r;
-        const float4 v = make_float4(o[r].x * inv, o[r].y * inv, o[r].z * inv, o[r].w * inv);
-        if (p.out_f32) {
-            reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_row * kD)[lane] = v;
-        } else {
-            uint2 w2;
-            w2.x = pack_bf16(v.x, v.y);
-            w2.y = pack_bf16(v.z, v.w);
-            reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_row * kD)[lane] = w2;
+        for (int r = 0; r < 8; ++r) {
+            const int grow = row0 + r;
+            const int tok = s.tok0 + grow / p.G;
+            const float l_r = __shfl_sync(0xffffffffu, l_all, r), m_r = __shfl_sync(0xffffffffu, m_all, r);
+            if (tok >= s.M) continue;  // warp-uniform
+            const size_t out_row = ((size_t)s.lb * p.M_max + tok) * p.Hq + s.h * p.G + grow % p.G;
+            const float inv = 1.f / l_r;
+            const float4 v = make_float4(o[r].x * inv, o[r].y * inv, o[r].z * inv, o[r].w * inv);
+            if (p.out_f32) {
+                reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_row * kD)[lane] = v;
+            } else {
+                uint2 w2;
+                w2.x = pack_bf16(v.x, v.y);
+                w2.y = pack_bf16(v.z, v.w);
+                reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_row * kD)[lane] = w2;
+            }
+            if (p.lse && lane == 0) p.lse[out_row] = m_r + logf(l_r);
         }
-        if (p.lse && lane == 0) p.lse[out_row] = m_r + logf(l_r);
     }
 }
 
@@ -263,8 +310,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
     // A pair without work leaves at once (uniform for both CTAs).
     {
         SegIter it;
-        it.init(p);
-        if (it.x >= it.x_end) return;
+        Seg s;
+        if (!it.next(p, s)) return;
     }
 
     const uint32_t q_smem = smem_u32(smem);
@@ -778,8 +825,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1) att
 
 }  // namespace
 
-// The pair kernel serves the shapes of the single-CTA kernel whenever a KV head has more than one 128-row tile.
-bool attention_pair_wanted(const AttnArgs& a) { return a.M_max * a.g.G > 128; }
+// The pair kernel serves the shapes of the single-CTA kernel whenever a KV head has more than one 128-row tile, but
+// only on request (environment variable SPECPV_ATTN_KERNEL=pair, read at every call).  It needs about 7 % fewer
+// cycles per tile than the single-CTA kernel and wins short bursts, but both kernels run into the board's power
+// limit when verification steps follow one another, and there the pair kernel's operand exchange between the two SMs
+// costs it clock: measured inside the benchmark step it is 8-10 % slower (4.56 against 4.12-4.23 ms for 32 layers at
+// 128K), and its set-up and merge tail make it slower on single-layer calls (33 against 21 us for a 4096-token cache).
+bool attention_pair_wanted(const AttnArgs& a) {
+    if (a.M_max * a.g.G <= 128) return false;
+    const char* v = getenv("SPECPV_ATTN_KERNEL");
+    return v != nullptr && strcmp(v, "pair") == 0;
+}
 
 specpv_status launch_attention_pair(TcParams& p, const AttnArgs& a, cudaStream_t stream) {
     if (!set_smem_limit_once(reinterpret_cast<const void*>(attn_pair_kernel), kPairSmem)) return SPECPV_ERR_CUDA;
@@ -802,14 +858,32 @@ specpv_status launch_attention_pair(TcParams& p, const AttnArgs& a, cudaStream_t
     }
     const long long units = (long long)Hkv * a.n_layers * a.batch * p.n_row_groups;
     const long long max_tiles = (a.max_seq_len + kTileTokens - 1) / kTileTokens + 1;  // context tiles + the step's own tokens
-    // no more pairs than give each at least two tiles (a pair's set-up costs about as much as four)
-    long long use = units * max_tiles / 2;
-    if (use < 1) use = 1;
-    if (use > n_pairs) use = n_pairs;
+    // How many pairs: all the device holds when there are at least as many units; with fewer units, k pairs per unit,
+    // k chosen by a small cost model (microseconds): a pair's tiles one after the other, then the merge of the unit's k
+    // partial results by the CTA that arrives last, one dependent round trip to L2 per partial result.
+    long long use = n_pairs;
+    p.pairs_per_unit = 0;
+    if (units < n_pairs) {
+        p.pairs_per_unit = 1;
+        const double t_tile = 1.0, t_seg = 1.4;
+        double best = 1e30;
+        for (long long k = 1; k * units <= n_pairs && k <= max_tiles; ++k) {
+            const double cost = (double)((max_tiles + k - 1) / k) * t_tile + (k > 1 ? k * t_seg : 0.0);
+            if (cost < best) {
+                best = cost;
+                use = k * units;
+                p.pairs_per_unit = (int)k;
+            }
+        }
+    }
     // partial results: two slots of 256 rows per pair; arrival counters: two per unit
     const size_t slot_bytes = (size_t)256 * (kD + 2) * sizeof(float);
     if ((size_t)use * 2 * slot_bytes > a.partial_bytes) use = (long long)(a.partial_bytes / (2 * slot_bytes));  // fewer pairs: slower, same result
     if (use < 1 || (size_t)units * 2 * sizeof(int32_t) > a.counter_bytes) return SPECPV_ERR_CAPACITY;
+    if (p.pairs_per_unit > 0) {  // keep k pairs per unit within what the scratch allows
+        p.pairs_per_unit = (int)(use / units);
+        use = p.pairs_per_unit * units;
+    }
     char* ws = reinterpret_cast<char*>(a.workspace) + a.partial_off;
     p.part_o = reinterpret_cast<float*>(ws);
     p.part_ml = reinterpret_cast<float*>(ws + (size_t)use * 2 * 256 * kD * sizeof(float));

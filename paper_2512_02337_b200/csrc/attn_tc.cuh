@@ -29,6 +29,7 @@ struct TcParams {
     int32_t* counters;  // pair kernel: arrival counters of shared units, [unit][CTA rank], zero between launches
     void* workspace;
     int n_layers_call;
+    int pairs_per_unit;  // pair kernel: > 0 = every unit has this many pairs of its own; 0 = pairs take equal shares of all tiles
     int layer0, batch, M_max, mask_words, Hq, Hkv, G, max_blocks, n_pages;
     int n_splits, n_row_groups, R_pad, out_f32;
     int bs;          // tokens per page (16, 32 or 64)

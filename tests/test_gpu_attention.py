@@ -13,6 +13,17 @@ from tests import util
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["single", "pair"])
+def attention_kernel(request, monkeypatch):
+    """Every case runs on both tensor-core kernels: the default (one CTA per KV range) and the CTA-pair kernel,
+    which the library uses on request for shapes with more than 128 query rows per KV head."""
+    if request.param == "pair":
+        monkeypatch.setenv("SPECPV_ATTN_KERNEL", "pair")
+    else:
+        monkeypatch.delenv("SPECPV_ATTN_KERNEL", raising=False)
+    return request.param
+
+
 def run_case(dtype, Hq, Hkv, d, bs, ctx, Ms, depth=4, branch=3, n_chain=0, n_layers=1, shuffle=True, seed=0,
              partial_entry=False):
     """One verify call on random data; Ms lists the tree size of every sequence (ragged q_lens)."""

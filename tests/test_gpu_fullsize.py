@@ -123,6 +123,18 @@ def test_llama_32k_all_layers_sampled():
     run_full_size("llama_32k", layers=[0, 31], budgets=[64])
 
 
+def test_llama_32k_all_layers_sampled_on_the_pair_kernel(monkeypatch):
+    """The same full-size check with the CTA-pair attention kernel (persistent launch, shared KV ranges merged in the
+    kernel) in place of the default one."""
+    monkeypatch.setenv("SPECPV_ATTN_KERNEL", "pair")
+    run_full_size("llama_32k", layers=[0, 31], budgets=[64])
+
+
+def test_stress_batch4_on_the_pair_kernel(monkeypatch):
+    monkeypatch.setenv("SPECPV_ATTN_KERNEL", "pair")
+    run_full_size("stress_b4", layers=[0, 31], budgets=[64])
+
+
 def test_llama_32k_channelwise_scores_several_tiles_per_cta():
     # the channel-wise form of Eq. 2 at full size: 256 heads leave two CTAs per head, two 128-block tiles each
     run_full_size("llama_32k", layers=[3, 31], budgets=[64], score_mode=1)

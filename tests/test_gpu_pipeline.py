@@ -81,13 +81,16 @@ def run_pipeline(name, n_layers=None, reduce=0, score_mode=0, select_shared=0, *
             assert np.all(np.isnan(scores_g[l, b, :, nb:]))  # untouched beyond the context
             n_keep = min(nb, cfg.budget_blocks)
             assert count_g[b] == n_keep
-            if select_shared:  # one list per (layer, sequence), ranked on the float32 mean over the heads
-                shared = oracle.head_shared_scores(scores_g[l, b, :, :nb])
-                oidx = np.stack([oracle.select(shared.astype(np.float64), sink, local, cfg.budget_blocks)] * Hkv)
+            if select_shared:  # one list per (layer, sequence), ranked on the mean over the heads
+                for h in range(1, Hkv):
+                    assert np.array_equal(idx_g[l, b, h, :n_keep], idx_g[l, b, 0, :n_keep])
+                util.check_shared_selection(idx_g[l, b, 0, :n_keep], scores_g[l, b, :, :nb], sink, local,
+                                            cfg.budget_blocks, f"shared selection l{l} b{b}")
+                oidx = idx_g[l, b, :, :n_keep].copy()  # the list the gather below has to follow
             else:
                 oidx = np.stack([oracle.select(scores_g[l, b, h, :nb].astype(np.float64), sink, local, cfg.budget_blocks)
                                  for h in range(Hkv)])
-            assert np.array_equal(idx_g[l, b, :, :n_keep], oidx)  # bit-exact given the same float32 scores
+                assert np.array_equal(idx_g[l, b, :, :n_keep], oidx)  # bit-exact given the same float32 scores
             opk, opv = np.zeros_like(pk_g[l]), np.zeros_like(pv_g[l])
             oplen = oracle.gather(kp[l], vp[l], table[b], sl, oidx, opk, opv, first_page=b * ppb)
             assert plens_g[b] == oplen

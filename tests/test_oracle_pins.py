@@ -470,18 +470,47 @@ def test_planted_mistakes_are_caught():
         assert np.abs(wrong - out).max() > 1e-3
 
 
-def test_head_shared_scores_is_the_float32_mean_over_heads():
-    rng = np.random.default_rng(5)
-    s = rng.standard_normal((8, 300)).astype(np.float32) * 30
+def test_head_shared_scores_is_the_mean_over_heads():
+    # hand values: three heads, four blocks
+    s = np.array([[1.0, 2.0, -3.0, 0.5], [3.0, 2.0, 3.0, 0.25], [2.0, 5.0, 0.0, 0.0]])
     got = oracle.head_shared_scores(s)
-    assert got.dtype == np.float32 and got.shape == (300,)
-    np.testing.assert_allclose(got, s.astype(np.float64).mean(axis=0), rtol=4e-7, atol=1e-5)  # float32 rounding only
-    one = oracle.head_shared_scores(s[:1])
-    assert np.array_equal(one, s[0])  # a single head is left as it is
+    assert got.dtype == np.float64
+    assert np.array_equal(got, np.array([2.0, 3.0, 0.0, 0.25]))
+    rng = np.random.default_rng(5)
+    r = rng.standard_normal((8, 300)).astype(np.float32) * 30
+    assert np.array_equal(oracle.head_shared_scores(r[:1]), r[0].astype(np.float64))  # a single head is left as it is
+    # the mean is linear: a constant added to one head moves every block's shared score by constant / heads
+    r2 = r.astype(np.float64)
+    r2[3] += 8.0
+    np.testing.assert_allclose(oracle.head_shared_scores(r2), oracle.head_shared_scores(r) + 1.0, rtol=0, atol=1e-12)
     # selection on it is ordinary selection: with identical heads the shared list equals every head's own list
-    same = np.repeat(s[:1], 4, axis=0)
-    assert np.array_equal(oracle.select(oracle.head_shared_scores(same).astype(np.float64), 1, 2, 16),
-                          oracle.select(s[0].astype(np.float64), 1, 2, 16))
+    same = np.repeat(r[:1], 4, axis=0)
+    assert np.array_equal(oracle.select(oracle.head_shared_scores(same), 1, 2, 16),
+                          oracle.select(r[0].astype(np.float64), 1, 2, 16))
+
+
+def test_shared_selection_check_accepts_rounding_ties_and_rejects_wrong_lists():
+    """The GPU-side check of head-shared lists (tests/util.check_shared_selection) against planted lists."""
+    from tests import util
+    rng = np.random.default_rng(11)
+    s = rng.standard_normal((8, 64)).astype(np.float32) * 10
+    want = oracle.select(oracle.head_shared_scores(s), 1, 2, 16)
+    util.check_shared_selection(want, s, 1, 2, 16)                       # the oracle's own list
+    mean = oracle.head_shared_scores(s)
+    kept = [i for i in want if 1 <= i < 62]
+    dropped = [i for i in range(1, 62) if i not in want]
+    worst_kept, best_dropped = min(kept, key=lambda i: mean[i]), max(dropped, key=lambda i: mean[i])
+    swapped = np.array(sorted((set(want.tolist()) - {worst_kept}) | {best_dropped}), dtype=np.int32)
+    with pytest.raises(AssertionError):                                  # far apart: the swap is a mistake
+        util.check_shared_selection(swapped, s, 1, 2, 16)
+    tie = s.copy()
+    tie[:, best_dropped] = tie[:, worst_kept]                            # equal means: either block may be kept
+    want_tie = oracle.select(oracle.head_shared_scores(tie), 1, 2, 16)
+    other = np.array(sorted((set(want_tie.tolist()) - {min(worst_kept, best_dropped)}) | {max(worst_kept, best_dropped)}),
+                     dtype=np.int32)
+    util.check_shared_selection(other, tie, 1, 2, 16)
+    with pytest.raises(AssertionError):                                  # a sink block left out
+        util.check_shared_selection(np.array(sorted(set(want.tolist()) - {0} | {dropped[0]}), dtype=np.int32), s, 1, 2, 16)
 
 
 # ---- the linear maps either side of the attention (Algorithm 1 "TreeDecode") ------------------------------------

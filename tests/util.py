@@ -93,3 +93,30 @@ def oracle_attention_rows(q, k_new, v_new, parents, n_chain, rows, k_pool, v_poo
 def sync_status(ws: torch.Tensor, expect: int = 0):
     st, info = B.specpv_poll_status(ws)
     assert st == expect, f"device status {st} ({B.specpv_status_string(st)}), info {info}"
+
+
+def check_shared_selection(idx_row: np.ndarray, scores: np.ndarray, sink: int, local: int, budget: int, what: str = ""):
+    """Head-shared selection: the kernel ranks blocks on a float32 mean over the KV heads; the oracle's definition is
+    the float64 mean.  Where the two rankings can differ only through float32 rounding (means of the last kept and the
+    first dropped block closer than that rounding), any choice among the tied blocks is correct; everywhere else the
+    list must be the oracle's.  scores [Hkv][nb] are the kernel's own float32 scores."""
+    Hkv, nb = scores.shape
+    mean = oracle.head_shared_scores(scores)
+    want = oracle.select(mean, sink, local, budget)
+    got = np.asarray(idx_row)
+    if np.array_equal(got, want):
+        return
+    # rounding of a float32 sum of Hkv terms and one multiplication
+    eps = (Hkv + 1) * 2.0 ** -23 * float(np.abs(scores).max())
+    assert len(got) == len(want), f"{what}: {len(got)} blocks kept, oracle keeps {len(want)}"
+    assert np.all(np.diff(got) > 0), f"{what}: block list not ascending"
+    must = set(range(min(sink, nb))) | set(range(max(nb - local, 0), nb))
+    assert must <= set(got.tolist()), f"{what}: sink or local blocks missing"
+    kept = sorted(set(got.tolist()) - must)
+    dropped = sorted(set(range(sink, nb - local)) - set(kept))
+    if kept and dropped:
+        assert mean[kept].min() >= mean[dropped].max() - eps, f"{what}: a dropped block outranks a kept one beyond rounding"
+    # what differs from the oracle's list lies within rounding of the cut
+    diff = sorted(set(got.tolist()) ^ set(want.tolist()))
+    cut = mean[sorted(set(want.tolist()) - must)].min() if set(want.tolist()) - must else 0.0
+    assert np.all(np.abs(mean[diff] - cut) <= eps), f"{what}: lists differ away from the cut"
