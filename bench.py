@@ -494,6 +494,12 @@ def score_variants(st, peaks, iters=10):
     return res
 
 
+def workload_string(name, c, n_layers, budget_tokens, batch):
+    """The `config.workload` text, the same in both arms."""
+    return (f"{name}: {n_layers} layers, Hq {c['Hq']}, Hkv {c['Hkv']}, d {c['d']}, ctx {c['ctx']}, {c['bs']}-token pages, "
+            f"tree {c['M']} nodes, budget {budget_tokens} tokens, batch {batch}")
+
+
 def algorithmic_work(st):
     """Bytes and flops of one full-verification launch: K/V actually attended + Q, O, Knew, Vnew."""
     c = st["w"].cfg
@@ -507,21 +513,17 @@ def algorithmic_work(st):
     return kv_bytes + step_bytes, flops, L * M * tokens
 
 
-def oracle_sample(st, budget_s=20.0):
-    """Time the CPU oracle (as it stands) on a bounded sample and scale to one step.
+def oracle_sample(st):
+    """Time the CPU oracle (as it stands) on one whole layer and scale by the layer count only.
 
-    Sample: layer 0, sequence 0, all KV heads, the rows of one root-to-leaf path of the tree, full
-    verification over the whole context plus partial verification over the partial cache; scaled by
-    (tree tokens / path tokens) x layers x sequences (by context share)."""
+    Sample: layer 0, sequence 0, all KV heads, ALL rows of the step: full verification over the whole context plus
+    partial verification over the partial cache; x layers, and for a batch x the sequences' share of the context."""
     import oracle
     w, c = st["w"], st["w"].cfg
-    B = st["B"]
     M = c["M"]
-    depth_of = [len(wl.path_to(w.parents[0], n)) for n in range(M)]
-    path = wl.path_to(w.parents[0], int(np.argmax(depth_of)))
     kp, vp = wl.to_numpy(w.k_pool[0]), wl.to_numpy(w.v_pool[0])
-    q, kn, vn = (wl.to_numpy(t[0, 0])[path] for t in (w.q, w.k_new, w.v_new))
-    mask = oracle.tree_mask(np.arange(-1, len(path) - 1, dtype=np.int32))
+    q, kn, vn = (wl.to_numpy(t[0, 0]) for t in (w.q, w.k_new, w.v_new))
+    mask = oracle.tree_mask(w.parents[0])
     table = w.block_table[0].cpu().numpy()
     sl = int(st["lens0"][0])
     t0 = time.perf_counter()
@@ -532,11 +534,10 @@ def oracle_sample(st, budget_s=20.0):
     t0 = time.perf_counter()
     oracle.tree_attention(q, kn, vn, mask, pk, pv, st["partial"].block_table[0].cpu().numpy(), plen)
     t_part = time.perf_counter() - t0
-    scale = (M / len(path)) * st["L"] * (sum(c["ctx"]) / c["ctx"][0])
-    us = (t_full * scale + t_part * (M / len(path)) * st["L"] * st["batch"]) * 1e6
-    sample = (f"layer 0, sequence 0, all {c['Hkv']} KV heads, {len(path)} of {M} tree tokens (one root-to-leaf "
-              f"path): full verify over {sl} tokens {t_full:.2f}s + partial verify over {plen} tokens "
-              f"{t_part:.2f}s; scaled x{M / len(path):.2f} tokens x{st['L']} layers x sequences; attention only")
+    us = (t_full * st["L"] * (sum(c["ctx"]) / c["ctx"][0]) + t_part * st["L"] * st["batch"]) * 1e6
+    sample = (f"one whole layer (layer 0, sequence 0, all {c['Hkv']} KV heads, all {M} step tokens): full verify over "
+              f"{sl} tokens {t_full:.2f}s + partial verify over {plen} tokens {t_part:.2f}s; x {st['L']} layers"
+              + (f" x sequences by context share" if st["batch"] > 1 else "") + "; attention only")
     return us, sample, oracle.num_threads()
 
 
@@ -641,9 +642,7 @@ def main():
         "metric": METRIC, "value": ms_step * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": c["dtype"], "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {st['L']} layers, Hq {c['Hq']}, Hkv {c['Hkv']}, d {c['d']}, "
-                               f"ctx {c['ctx']}, {c['bs']}-token pages, tree {c['M']} nodes, budget "
-                               f"{st['cfg'].budget_blocks * c['bs']} tokens, batch {st['batch']}",
+        "config": {"workload": workload_string(args.workload, c, st["L"], st["cfg"].budget_blocks * c["bs"], st["batch"]),
                    "step": "refresh step (full verify + commit + scores + select + gather) + partial step "
                            "(partial verify + commit)",
                    "l2": "inputs larger than L2 (every step streams all layers' caches)",
@@ -677,35 +676,38 @@ def main():
 
 
 def reference_arm(args):
-    """Times the CPU oracle, as it stands, on bounded samples of the workload (no GPU work at all)."""
+    """Times the CPU oracle, as it stands, on the default arm's workload (no GPU work at all).  A step of this arm is
+    a bounded sample of the workload's step: one whole layer of sequence 0 (all KV heads, all step tokens, the uncut
+    context) through full verification and through partial verification over a cache of the budget's length; the
+    value is that time x layers (x the sequences' share of the context for a batch)."""
     import oracle
     name = args.workload
     c = dict(wl.CONFIGS[name])
-    # one layer, a cut of the context: the sample is scaled to the full step below
-    ctx_cut = [min(x, 8192) for x in c["ctx"]]
-    w = wl.make_workload(name, device="cpu", n_layers=1, ctx=ctx_cut)
+    n_layers = args.layers or c["n_layers"]
+    w = wl.make_workload(name, device="cpu", n_layers=1, ctx=[c["ctx"][0]])
     M = c["M"]
-    depth_of = [len(wl.path_to(w.parents[0], n)) for n in range(M)]
-    path = wl.path_to(w.parents[0], int(np.argmax(depth_of)))
     kp, vp = wl.to_numpy(w.k_pool[0]), wl.to_numpy(w.v_pool[0])
-    q, kn, vn = (wl.to_numpy(t[0, 0])[path] for t in (w.q, w.k_new, w.v_new))
-    mask = oracle.tree_mask(np.arange(-1, len(path) - 1, dtype=np.int32))
+    q, kn, vn = (wl.to_numpy(t[0, 0]) for t in (w.q, w.k_new, w.v_new))
+    mask = oracle.tree_mask(w.parents[0])
     table = w.block_table[0].numpy()
+    budget = (args.budget_blocks or c["budget_blocks"]) * c["bs"]
     times = []
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        oracle.tree_attention(q, kn, vn, mask, kp, vp, table, ctx_cut[0])
+        oracle.tree_attention(q, kn, vn, mask, kp, vp, table, c["ctx"][0])   # full verification, one layer
+        oracle.tree_attention(q, kn, vn, mask, kp, vp, table, budget)        # partial verification: a cache of the budget's length
         if i >= args.warmup:
             times.append(time.perf_counter() - t0)
-    budget = c["budget_blocks"] * c["bs"]
-    per_token_row = statistics.mean(times) / (ctx_cut[0] + len(path)) / len(path)
-    step_s = per_token_row * M * c["n_layers"] * (sum(c["ctx"]) + len(c["ctx"]) * budget)
-    sample = (f"oracle attention, 1 layer, sequence 0 cut to {ctx_cut[0]} tokens, all KV heads, {len(path)} of {M} "
-              f"tree tokens; scaled linearly in tokens x rows x layers to the full and partial verification of a step")
+    batch = len(c["ctx"])
+    layer_s = statistics.mean(times)
+    step_s = layer_s * n_layers * (sum(c["ctx"]) + batch * budget) / (c["ctx"][0] + budget)
+    sample = (f"oracle attention of one whole layer per step (sequence 0, all {c['Hkv']} KV heads, all {M} step tokens): full "
+              f"verify over {c['ctx'][0]} tokens + partial verify over {budget} tokens, {layer_s:.2f}s; x {n_layers} layers"
+              + (" x sequences by context share" if batch > 1 else ""))
     out = {"impl": "reference", "metric": METRIC, "value": step_s * 1e6, "unit": "us", "n_gpus": 1,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": False,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"{name} (see the default arm)"},
+           "config": {"workload": workload_string(name, c, n_layers, budget, batch)},
            "cpu_baseline": {"value": step_s * 1e6, "unit": "us", "cores": oracle.num_threads(), "kind": "oracle",
                             "sample": sample},
            "e2e": {"value": step_s * 1e6, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}

@@ -31,6 +31,10 @@ EXPORTS = [
 ]
 
 
+SELFTEST_EXPORTS = ["specpv_selftest_wait_timeout"]  # include/specpv_selftest.h
+SELFTEST_WHERE = 99
+
+
 class SpecPVError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -69,7 +73,7 @@ def lib() -> ctypes.CDLL:
         _lib.specpv_workspace_bytes.restype = c_size_t
         _lib.specpv_workspace_bytes.argtypes = [POINTER(Config), c_int, c_int, c_int, c_int]
         _lib.specpv_kernel_launches.restype = ctypes.c_uint64
-        for name in EXPORTS[3:]:
+        for name in EXPORTS[3:] + SELFTEST_EXPORTS:
             getattr(_lib, name).restype = c_int
     return _lib
 
@@ -224,6 +228,14 @@ def specpv_verify_partial_static(cfg, layer0, n_layers, q, k_new, v_new, tree_ma
                                               _ptr(tree_mask), _ptr(q_lens), M_max, ctypes.byref(d), _ptr(out),
                                               _ptr(lse), _ptr(device_status), _stream(stream)),
            "specpv_verify_partial_static")
+
+
+def specpv_selftest_wait_timeout(workspace, limit_us: int, observed_ns=None, stream=None):
+    """Self-test (include/specpv_selftest.h): a bounded barrier wait that runs out after ``limit_us`` microseconds and
+    records SPECPV_ERR_TIMEOUT in the workspace's status word.  ``observed_ns``: optional uint64/int64 device tensor."""
+    _check(lib().specpv_selftest_wait_timeout(_ptr(workspace), c_size_t(workspace.numel() * workspace.element_size()),
+                                              int(limit_us), _ptr(observed_ns), _stream(stream)),
+           "specpv_selftest_wait_timeout")
 
 
 def specpv_verify_full(cfg, layer0, n_layers, q, k_new, v_new, tree_mask, q_lens, M_max, full: Cache, out, lse,

@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "lib" / "libspecpv.so"
-SOURCES = ["api.cu", "aux_kernels.cu", "attn_simt.cu", "attn_tc.cu", "attn_pair.cu", "score_tc.cu", "proj_tc.cu", "offload.cu"]
+SOURCES = ["api.cu", "aux_kernels.cu", "attn_simt.cu", "attn_tc.cu", "attn_pair.cu", "score_tc.cu", "proj_tc.cu", "offload.cu", "selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-fvisibility=hidden",

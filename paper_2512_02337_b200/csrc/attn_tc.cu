@@ -46,6 +46,7 @@ struct __align__(8) Barriers {
     uint64_t o_done[2];         // the last PV of row tile t has completed
     uint64_t v_need;            // MMA issuer -> warp 2: this V tile has landed and needs its tail rows zeroed
     uint64_t v_fixed;           // warp 2 -> MMA issuer: done
+    uint64_t drain;             // completion of the contractions issued before a wait gave up
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -114,6 +115,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         }
         mbar_init(smem_u32(&bars.v_need), 1);
         mbar_init(smem_u32(&bars.v_fixed), 1);
+        mbar_init(smem_u32(&bars.drain), 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -131,7 +133,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
 
     // Register budget: the control warpgroup (warps 0-3) gives registers to the two softmax warpgroups.
     if (warp == 0) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         // =========================== TMA producer ================================================
         // The whole warp runs the loop (a lone lane of a diverged warp runs slowly); lane 0 issues the copies.
         const uint32_t qbar = smem_u32(&bars.q_full);
@@ -172,7 +174,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             row_next = page_row(j + 1);
             for (int kv = 0; kv < 2; ++kv) {  // 0: K tile, 1: V tile
                 const uint32_t full = smem_u32(&bars.kv_full[slot]), empty = smem_u32(&bars.kv_empty[slot]);
-                if (2 * j + kv >= kStages) ok &= mbar_wait(empty, par, abort_flag, p.workspace, 1);
+                if (2 * j + kv >= kStages) ok = mbar_wait(empty, par, abort_flag, p.workspace, 1);
+                if (!ok) break;  // a wait gave up: nothing more is copied
                 const uint32_t dst = kv_smem + slot * kSlotBytes + my_half * 16384;
                 if (lane == 0) mbar_expect_tx(full, kSlotBytes);
                 if (is_new) {  // the step's own tokens: two boxes of 64 rows per half
@@ -185,10 +188,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 __syncwarp();
                 if (++slot == kStages) { slot = 0; par ^= 1; }
             }
+            if (!ok) break;
         }
-        (void)ok;
     } else if (warp == 1) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         // =========================== MMA issuer ==================================================
         // One warp issues every contraction (issuing from two warps serialises the tensor pipe).  Issue
         // order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | ...
@@ -208,20 +211,23 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         uint32_t k_slot = 0, k_par = 0, v_slot = 1, v_par = 0;
         for (int j = 0; j <= n_tiles; ++j) {
             const int jp = j - 1;
-            if (j < n_tiles) ok &= mbar_wait(full0 + k_slot * 8, k_par, abort_flag, p.workspace, 3);
-            if (j > 0) {
-                ok &= mbar_wait(full0 + v_slot * 8, v_par, abort_flag, p.workspace, 4);
+            // a wait that gives up ends the loop: nothing more is issued (every lane sees the same result of a wait)
+            if (ok && j < n_tiles) ok = mbar_wait(full0 + k_slot * 8, k_par, abort_flag, p.workspace, 3);
+            if (ok && j > 0) {
+                ok = mbar_wait(full0 + v_slot * 8, v_par, abort_flag, p.workspace, 4);
                 // a ragged or tree tile: warp 2 zeroes the rows of V past the valid tokens first
-                if (jp >= first_fix) {
+                if (ok && jp >= first_fix) {
                     if (lane == 0) mbar_arrive(smem_u32(&bars.v_need));
-                    ok &= mbar_wait(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, abort_flag, p.workspace, 9);
+                    ok = mbar_wait(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, abort_flag, p.workspace, 9);
                 }
             }
+            if (!ok) break;
             const uint32_t kb_lo = launder(k_lo0 + k_slot * (kSlotBytes >> 4));
             const uint32_t vb_lo = launder(v_lo0 + v_slot * (kSlotBytes >> 4));
             for (int t = 0; t < n_q_tiles; ++t) {
                 if (j > 0) {
-                    ok &= mbar_wait(pfull0 + t * 8, jp & 1, abort_flag, p.workspace, 5);
+                    ok = mbar_wait(pfull0 + t * 8, jp & 1, abort_flag, p.workspace, 5);
+                    if (!ok) break;
                     tc_fence_after();
                 }
                 if (lane == 0) {
@@ -248,12 +254,20 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 }
                 __syncwarp();
             }
+            if (!ok) break;
             if (j < n_tiles) { k_slot += 2; if (k_slot >= kStages) { k_slot -= kStages; k_par ^= 1; } }
             if (j > 0) { v_slot += 2; if (v_slot >= kStages) { v_slot -= kStages; v_par ^= 1; } }
         }
-        (void)ok;
+        if (!ok && lane == 0) {
+            // after a give-up: wait (bounded) until the contractions that WERE issued have completed, so that the
+            // tensor memory is not freed under them
+            tc_commit(smem_u32(&bars.drain));
+            const uint64_t t0 = global_ns();
+            while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < 100000000ull) {}
+        }
+        __syncwarp();
     } else if (warp == 2) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         // =========================== V fixer =====================================================
         // Rows of a V tile past its valid tokens may hold anything (stale shared memory, rows of other
         // sequences' steps): zero them so that 0 * garbage cannot produce NaN.  Only the last context
@@ -276,9 +290,9 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             if (lane == 0) mbar_arrive(smem_u32(&bars.v_fixed));
         }
     } else if (warp == 3) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // =========================== softmax / correction / epilogue ==============================
         const int t = (warp - 4) >> 2;           // row tile of this warpgroup
         const int q = warp & 3;                  // TMEM lane quarter this warp may access
@@ -484,7 +498,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        if (*abort_flag) __nanosleep(200000);  // let copies in flight land before the CTA goes away
+        // after a give-up no new copy was issued; the few in flight (at most a ring of them) land within microseconds
+        if (*abort_flag) __nanosleep(1000000);
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }

@@ -26,10 +26,7 @@ constexpr int kWTileBytes = kFeatTile * 128;  // 128 features x 64 input feature
 constexpr int kProjDataBytes = 192 * 1024;
 constexpr int kProjSmem = 1024 + kProjDataBytes;
 constexpr int kProjMaxStages = 8;
-#ifndef PROJ_ISSUE_GROUP
-#define PROJ_ISSUE_GROUP 2
-#endif
-constexpr int kIssueGroup = PROJ_ISSUE_GROUP;  // stages whose copies are issued together
+constexpr int kIssueGroup = 2;             // stages whose copies are issued together
 constexpr int kMaxTokTile = 256;           // rows per CTA (accumulator columns)
 
 struct ProjTcParams {
@@ -130,7 +127,8 @@ __global__ void __launch_bounds__(kProjThreads, 2) proj_tc_kernel(const __grid_c
             for (int i = i0; i < i1; ++i)
                 if (i >= p.stages)
                     ok &= mbar_wait(smem_u32(&bars.empty[i % p.stages]), ((i / p.stages) - 1) & 1, abort_flag, p.workspace, 30);
-            if (lane == 0 && ok) {
+            if (!ok) break;  // a wait gave up: nothing more is copied
+            if (lane == 0) {
                 for (int i = i0; i < i1; ++i) {
                     const int slot = i % p.stages;
                     const uint32_t full = smem_u32(&bars.full[slot]);
@@ -150,8 +148,9 @@ __global__ void __launch_bounds__(kProjThreads, 2) proj_tc_kernel(const __grid_c
         for (int i = 0; i < n_k; ++i) {
             const int slot = i % p.stages;
             ok &= mbar_wait(smem_u32(&bars.full[slot]), (i / p.stages) & 1, abort_flag, p.workspace, 31);
+            if (!ok) break;  // a wait gave up: nothing more is issued
             tc_fence_after();
-            if (lane == 0 && ok) {
+            if (lane == 0) {
                 const uint32_t a_lo = (((data + slot * stage_bytes) >> 4) & 0x3FFFu) | (1u << 16);
                 const uint32_t b_lo = (((data + slot * stage_bytes + kWTileBytes) >> 4) & 0x3FFFu) | (1u << 16);
 #pragma unroll
@@ -200,7 +199,8 @@ __global__ void __launch_bounds__(kProjThreads, 2) proj_tc_kernel(const __grid_c
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        if (*abort_flag) __nanosleep(200000);
+        // after a give-up nothing new was issued; the few copies and contractions in flight end within microseconds
+        if (*abort_flag) __nanosleep(1000000);
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
     }

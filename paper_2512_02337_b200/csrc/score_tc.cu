@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
             const int slot = i % stages;
             ok &= mbar_wait(smem_u32(&bars.sum_full[slot]), (i / stages) & 1, abort_flag, p.workspace, 22);
             if (i > 0) ok &= mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
+            if (!ok) break;  // a wait gave up: nothing more is copied or issued
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t a_max = sum_lo + (uint32_t)slot * (2 * kSumTileBytes >> 4), a_min = a_max + (kSumTileBytes >> 4);
@@ -284,7 +285,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        if (*abort_flag) __nanosleep(200000);
+        // after a give-up nothing new was issued; the few copies and contractions in flight end within microseconds
+        if (*abort_flag) __nanosleep(1000000);
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }

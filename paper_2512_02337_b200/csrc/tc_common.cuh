@@ -58,15 +58,16 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 
-// Bounded wait: gives up after about two seconds (or when another thread already gave up), records
+// Bounded wait: gives up after `limit_ns` (or when another thread of the CTA already gave up), records
 // SPECPV_ERR_TIMEOUT and raises the CTA's abort flag.  Returns false on give-up.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // the product kernels' limit: two seconds
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
-                                            int where) {
+                                            int where, uint64_t limit_ns) {
     const uint64_t t0 = global_ns();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((it & 255u) == 255u && global_ns() - t0 > 2000000000ull) {
+        if ((it & 255u) == 255u && global_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             record_fault(workspace, SPECPV_ERR_TIMEOUT, where, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
             return false;
@@ -74,9 +75,9 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, vo
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, void* workspace,
-                                          int where) {
+                                          int where, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, workspace, where);
+    return mbar_wait_slow(bar, parity, abort_flag, workspace, where, limit_ns);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {

@@ -186,6 +186,34 @@ def test_commit_appends_and_updates_summaries():
     assert torch.equal(kmax[:, :, :, :nb], kmax2[:, :, :, :nb]) and torch.equal(kmin[:, :, :, :nb], kmin2[:, :, :, :nb])
 
 
+def test_commit_in_layer_groups_matches_the_oracle():
+    """A step's commit issued in two layer groups, in ascending order: every group writes its rows at the lengths as
+    they stand and the lengths advance with the group that holds the model's last layer."""
+    w = wl.make_workload("llama_32k", device="cuda", n_layers=3, spare_tokens=64, ctx=[64 * 20 + 9], M=20)
+    c = w.cfg
+    L, M = c["n_layers"], c["M"]
+    cfg = util.config_for(w)
+    full = util.full_cache(w)
+    ws = B.new_workspace(cfg, L, 1, int(max(c["ctx"])) + 64, M)
+    path = wl.path_to(w.parents[0], int(np.argmax([len(wl.path_to(w.parents[0], n)) for n in range(M)])))
+    acc = torch.zeros((1, 8), dtype=torch.int32, device="cuda")
+    acc[0, :len(path)] = torch.from_numpy(path).cuda()
+    n_acc = torch.tensor([len(path)], dtype=torch.int32, device="cuda")
+    kp0, vp0 = wl.to_numpy(w.k_pool).copy(), wl.to_numpy(w.v_pool).copy()
+    sl0 = int(w.seq_lens[0])
+    B.specpv_commit_accepted(cfg, 0, 2, w.k_new[0:2], w.v_new[0:2], M, acc, n_acc, 8, full, None, None, ws)
+    torch.cuda.synchronize()
+    assert int(w.seq_lens[0]) == sl0                      # not yet: the last layer is not in this group
+    B.specpv_commit_accepted(cfg, 2, 1, w.k_new[2:3], w.v_new[2:3], M, acc, n_acc, 8, full, None, None, ws)
+    util.sync_status(ws)
+    assert int(w.seq_lens[0]) == sl0 + len(path)
+    table = w.block_table.cpu().numpy()
+    knn, vnn = wl.to_numpy(w.k_new), wl.to_numpy(w.v_new)
+    for l in range(L):
+        assert oracle.commit(knn[l, 0], vnn[l, 0], path, kp0[l], vp0[l], table[0], sl0) == sl0 + len(path)
+    assert np.array_equal(wl.to_numpy(w.k_pool), kp0) and np.array_equal(wl.to_numpy(w.v_pool), vp0)
+
+
 @pytest.mark.parametrize("nb,budget", [(300, 40), (2048, 64), (4099, 128), (9000, 1000)])
 def test_selection_alone_on_synthetic_scores_with_ties_and_nan(nb, budget):
     """The selection kernel on its own: more candidate blocks than it keeps in registers (nb > 4096), repeated

@@ -25,8 +25,11 @@ def test_library_exports_every_declared_symbol():
     header = (ROOT / "include" / "specpv.h").read_text()
     declared = set(re.findall(r"\b(specpv_[a-z_0-9]+)\s*\(", header))
     assert declared == set(B.EXPORTS)
+    selftest = (ROOT / "include" / "specpv_selftest.h").read_text()
+    declared_selftest = set(re.findall(r"\b(specpv_[a-z_0-9]+)\s*\(", selftest))
+    assert declared_selftest == set(B.SELFTEST_EXPORTS)
     lib = B.lib()
-    for name in declared:
+    for name in declared | declared_selftest:
         assert getattr(lib, name) is not None
 
 
