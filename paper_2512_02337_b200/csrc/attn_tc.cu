@@ -196,8 +196,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         // One warp issues every contraction (issuing from two warps serialises the tensor pipe).  Issue
         // order (ping-pong of the two row tiles): QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | ...
         // Barrier instructions do not overlap with queued MMAs (each costs the pipe 30-100 idle cycles),
-        // so the loop keeps them to four waits per KV tile, without votes, and four commits behind MMAs.  The whole warp runs the loop, lane 0 issues.  A wait that gives up makes
-        // every later wait return at once (abort flag), so the loop simply runs out.
+        // so the loop keeps them to four waits per KV tile, without votes, and four commits behind MMAs.  The whole
+        // warp runs the loop, lane 0 issues.
         bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 2));
         // Shared-memory descriptors: the upper word (stride between 8-row groups, version, swizzle) is
         // constant; the lower word is the 16-byte address plus the leading-dimension offset.
@@ -211,23 +211,23 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         uint32_t k_slot = 0, k_par = 0, v_slot = 1, v_par = 0;
         for (int j = 0; j <= n_tiles; ++j) {
             const int jp = j - 1;
-            // a wait that gives up ends the loop: nothing more is issued (every lane sees the same result of a wait)
-            if (ok && j < n_tiles) ok = mbar_wait(full0 + k_slot * 8, k_par, abort_flag, p.workspace, 3);
-            if (ok && j > 0) {
-                ok = mbar_wait(full0 + v_slot * 8, v_par, abort_flag, p.workspace, 4);
+            // A wait that gives up raises the abort flag, which makes the later waits of this tile return at once; the
+            // loop ends after this tile, so at most one tile's contractions are issued past the failed wait.  (One exit
+            // per tile: an exit after every wait costs the issuing thread 7 % of the kernel.)
+            if (j < n_tiles) ok &= mbar_wait(full0 + k_slot * 8, k_par, abort_flag, p.workspace, 3);
+            if (j > 0) {
+                ok &= mbar_wait(full0 + v_slot * 8, v_par, abort_flag, p.workspace, 4);
                 // a ragged or tree tile: warp 2 zeroes the rows of V past the valid tokens first
-                if (ok && jp >= first_fix) {
+                if (jp >= first_fix) {
                     if (lane == 0) mbar_arrive(smem_u32(&bars.v_need));
-                    ok = mbar_wait(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, abort_flag, p.workspace, 9);
+                    ok &= mbar_wait(smem_u32(&bars.v_fixed), (jp - first_fix) & 1, abort_flag, p.workspace, 9);
                 }
             }
-            if (!ok) break;
             const uint32_t kb_lo = launder(k_lo0 + k_slot * (kSlotBytes >> 4));
             const uint32_t vb_lo = launder(v_lo0 + v_slot * (kSlotBytes >> 4));
             for (int t = 0; t < n_q_tiles; ++t) {
                 if (j > 0) {
-                    ok = mbar_wait(pfull0 + t * 8, jp & 1, abort_flag, p.workspace, 5);
-                    if (!ok) break;
+                    ok &= mbar_wait(pfull0 + t * 8, jp & 1, abort_flag, p.workspace, 5);
                     tc_fence_after();
                 }
                 if (lane == 0) {
