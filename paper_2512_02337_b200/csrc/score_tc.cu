@@ -7,12 +7,22 @@
 //
 // Per (layer, sequence, KV head) the two products are dense contractions
 //     Dmax[128 blocks x R] = Kmax_tile[128 x 128] * Q^T[128 x R],   Dmin likewise with Kmin,
-// issued as tcgen05.mma with both operands in shared memory (128-byte swizzle, loaded by TMA) and
-// float32 accumulators in tensor memory (Dmax in columns [0, 256), Dmin in [256, 512)).  A CTA owns a
-// run of 128-block tiles of one head; thread i of the 128 epilogue threads owns block i of the tile
-// (tensor-memory lane i), takes max(Dmax, Dmin) per query row and reduces over the rows (mean, max,
-// or the rows of the "last" query).  The summaries of the next tile are in flight while a tile is
-// reduced.  Every wait is bounded.
+// issued as tcgen05.mma with both operands in shared memory (128-byte swizzle, loaded by TMA) and float32
+// accumulators in tensor memory.
+//
+// The kernel is persistent: one CTA per SM takes an equal contiguous share of all 128-block tiles of the launch
+// (layer-major, then sequence, KV head, tile), so a CTA sets up once and reloads Q only where its share crosses
+// into another head.  Tensor memory holds two accumulator regions of 256 columns (one per query row): Dmax in the
+// first, Dmin in the second.  Each product has its own issuing warp and its own stream of ring slots, so the barrier
+// work of one overlaps the contractions of the other, and a region is free again as soon as the epilogue has READ it:
+// Dmax is read into registers while the Dmin contractions run, the next tile's Dmax contractions run while the
+// epilogue takes max(Dmax, Dmin) and reduces.  The tensor pipe never waits for the reduction.  (The channel-wise form
+// has one accumulator per tile, so its tiles simply alternate between the two regions and the two issuing warps.)
+//   warp 0      TMA producer: Q of a head, then per tile its Kmax rows and its Kmin rows through a ring of 32 KB slots
+//   warps 1, 2  MMA issue: Dmax / Dmin (warp 1 also allocates the tensor memory)
+//   warps 4-11  epilogue: thread <-> block of the tile (tensor-memory lane) and one half of the query rows; reduces
+//               over its rows (mean, max, or the rows of the "last" query); the two halves meet in shared memory
+// Every wait is bounded; after a wait that gave up the loops end and nothing more is copied or issued.
 #include "aux_kernels.cuh"
 #include "tc_common.cuh"
 
@@ -22,18 +32,13 @@ namespace {
 
 using namespace tc;
 
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-constexpr int kScoreThreads = 192;       // warp 0: TMA + MMA issue, warp 1: idle, warps 2-5: epilogue (lane quarters 2,3,0,1)
+constexpr int kScoreThreads = 384;       // 12 warps; the four control warps hand registers to the eight epilogue warps
+constexpr int kScoreCtas = 148;          // one per SM
 constexpr int kTileBlocks = 128;
-constexpr int kSumTileBytes = 32768;     // [2 d-halves][128 blocks][64 d] bf16
-constexpr int kScoreStages = 2;
+constexpr int kSumTileBytes = 32768;     // a ring slot: the Kmax or the Kmin rows of a tile, [2 d-halves][128 blocks][64 d] bf16
+constexpr int kScoreStages = 5;          // ring slots (the channel-wise form gives two of them to q-)
 constexpr int kScoreQBytes = 65536;      // [2 d-halves][256 rows][64 d] bf16
-constexpr int kScoreSmem = 1024 + kScoreQBytes + kScoreStages * 2 * kSumTileBytes;
+constexpr int kScoreSmem = 1024 + kScoreQBytes + kScoreStages * kSumTileBytes;
 
 struct ScoreTcParams {
     CUtensorMap tm_q;     // (d, Hq, tokens)  box (64, G, 128/G)
@@ -44,69 +49,105 @@ struct ScoreTcParams {
     const int32_t* seq_lens;
     float* scores;
     void* workspace;
-    int layer0, batch, M_max, Hkv, G, bs, max_blocks, reduce, tiles_per_cta, n_cols;
+    int layer0, batch, M_max, Hkv, G, bs, max_blocks, reduce, n_cols;
+    int tiles_max;    // tiles per head of the longest sequence: the launch's work is n_heads * tiles_max tile positions
+    int n_heads;      // layers of the call * sequences * KV heads
     int tok0, tok_n;  // this pass covers step tokens [tok0, tok0 + tok_n): 256 query rows at most (the accumulator's columns)
     int accumulate;   // a later pass: combine with the scores the earlier passes left
 };
 
 struct __align__(8) ScoreBarriers {
-    uint64_t q_full;
+    uint64_t q_full;                   // Q of a head has landed
+    uint64_t q_empty;                  // the last contraction that reads this Q has completed
+    uint64_t q_split;                  // channel-wise form: the eight epilogue warps have split Q by sign
     uint64_t sum_full[kScoreStages];
     uint64_t sum_empty[kScoreStages];
-    uint64_t d_full;
-    uint64_t d_empty;
-    uint64_t q_split;  // channel-wise form: the epilogue warps have split Q by sign
+    uint64_t r_full[2];                // per accumulator region: the contractions of a tile are complete
+    uint64_t r_empty[2];               // ... and the eight epilogue warps have read the region
+    uint64_t x_full[2];                // the warps of the upper half of the query rows have left their partial results (tile parity)
     uint32_t tmem_base;
     int abort_flag;
 };
 
-// kCw: the channel-wise form (a compile-time switch, so that the printed form's code is exactly what it was).
+// A stretch of tiles of one head that a CTA works on.
+struct ScoreSeg {
+    int lb, b, l, h;
+    int t0, t1;                      // tiles [t0, t1) of the head
+    int nb;                          // blocks of the sequence
+    int col_begin, col_end, denom;   // query rows (accumulator columns) that count, and what the mean divides by
+};
+
+// Walks a CTA's share [x, x_end) of the launch's tile positions head by head.  Lengths live on the device, so every
+// role works the stretches out for itself; all of them see the same sequence.
+struct ScoreIter {
+    long long x, x_end;
+    __device__ void init(const ScoreTcParams& p) {
+        const long long total = (long long)p.n_heads * p.tiles_max;
+        x = total * blockIdx.x / gridDim.x;
+        x_end = total * (blockIdx.x + 1) / gridDim.x;
+    }
+    __device__ bool next(const ScoreTcParams& p, ScoreSeg& s) {
+        while (x < x_end) {
+            const long long head = x / p.tiles_max;
+            const long long stop = min(x_end, (head + 1) * p.tiles_max);
+            s.t0 = (int)(x - head * p.tiles_max);
+            x = stop;
+            s.h = (int)(head % p.Hkv);
+            s.lb = (int)(head / p.Hkv);
+            s.b = s.lb % p.batch;
+            s.l = s.lb / p.batch;
+            const int seq_len = max(p.seq_lens[s.b], 0);
+            s.nb = min((seq_len + p.bs - 1) / p.bs, p.max_blocks);
+            s.t1 = min((int)(stop - head * p.tiles_max), (s.nb + kTileBlocks - 1) / kTileBlocks);
+            int M = p.q_lens ? p.q_lens[s.b] : p.M_max;
+            M = min(max(M, 0), p.M_max);
+            // query rows r = token * G + head of this pass's tokens, one accumulator column each
+            s.col_begin = 0;
+            s.col_end = min(max(M - p.tok0, 0), p.tok_n) * p.G;
+            s.denom = M * p.G;  // rows the mean runs over (all passes together)
+            if (p.reduce == SPECPV_REDUCE_LAST) {
+                int last = p.last_query ? p.last_query[s.b] : 0;
+                last = min(max(last, 0), max(M - 1, 0));
+                if (M <= 0 || last < p.tok0 || last >= p.tok0 + p.tok_n) continue;  // another pass holds that row
+                s.col_begin = (last - p.tok0) * p.G;
+                s.col_end = s.col_begin + p.G;
+                s.denom = p.G;
+            }
+            if (s.col_end > s.col_begin && s.t1 > s.t0) return true;
+        }
+        return false;
+    }
+};
+
+// kCw: the channel-wise form (a compile-time switch).
 template <bool kCw>
 __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __grid_constant__ ScoreTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ ScoreBarriers bars;
+    __shared__ float xch[2][kTileBlocks];  // partial results of the upper half of the query rows, by tile parity
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y, lb = blockIdx.z;
-    const int b = lb % p.batch, l = lb / p.batch;
-    const int seq_len = max(p.seq_lens[b], 0);
-    const int nb = min((seq_len + p.bs - 1) / p.bs, p.max_blocks);
-    const int tile_begin = blockIdx.x * p.tiles_per_cta;
-    const int tile_end = min(tile_begin + p.tiles_per_cta, (nb + kTileBlocks - 1) / kTileBlocks);
-    if (tile_begin >= tile_end) return;
-    const int n_tiles = tile_end - tile_begin;
-    int M = p.q_lens ? p.q_lens[b] : p.M_max;
-    M = min(max(M, 0), p.M_max);
-    // query rows r = token * G + head of this pass's tokens, one accumulator column each
-    int col_begin = 0, col_end = min(max(M - p.tok0, 0), p.tok_n) * p.G;
-    int denom = M * p.G;  // rows the mean runs over (all passes together)
-    if (p.reduce == SPECPV_REDUCE_LAST) {
-        int last = p.last_query ? p.last_query[b] : 0;
-        last = min(max(last, 0), max(M - 1, 0));
-        if (M <= 0 || last < p.tok0 || last >= p.tok0 + p.tok_n) return;  // another pass holds that row
-        col_begin = (last - p.tok0) * p.G;
-        col_end = col_begin + p.G;
-        denom = p.G;
-    }
-    if (col_end <= col_begin) return;
-    const bool combine = p.accumulate && p.reduce != SPECPV_REDUCE_LAST;
 
     const uint32_t q_smem = smem_u32(smem);
-    // channel-wise form: q- takes the place of the second summary stage, the summaries go through a single stage
-    constexpr int stages = kCw ? 1 : kScoreStages;
+    // channel-wise form: q- takes the place of two ring slots
+    constexpr int stages = kCw ? kScoreStages - 2 : kScoreStages;
     const uint32_t qneg_smem = q_smem + kScoreQBytes;
     const uint32_t sum_smem = q_smem + (kCw ? 2 : 1) * kScoreQBytes;
     volatile int* abort_flag = &bars.abort_flag;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 2);  // both issuing warps
+        mbar_init(smem_u32(&bars.q_split), 8);  // one arrival per epilogue warp
         for (int s = 0; s < kScoreStages; ++s) {
             mbar_init(smem_u32(&bars.sum_full[s]), 1);
             mbar_init(smem_u32(&bars.sum_empty[s]), 1);
         }
-        mbar_init(smem_u32(&bars.d_full), 1);
-        mbar_init(smem_u32(&bars.d_empty), 4);  // one arrival per epilogue warp
-        mbar_init(smem_u32(&bars.q_split), 4);
+        for (int r = 0; r < 2; ++r) {
+            mbar_init(smem_u32(&bars.r_full[r]), 1);
+            mbar_init(smem_u32(&bars.r_empty[r]), 8);
+            mbar_init(smem_u32(&bars.x_full[r]), 4);
+        }
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -121,164 +162,261 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     tc_fence_after();
     const uint32_t tmem = bars.tmem_base;
     const int tok_per_tile = 128 / p.G;
-    const uint32_t idesc = make_idesc((uint32_t)p.n_cols, false);
 
+    // Register budget: 384 threads start with 168 registers each; the control warps keep 48, which is what lets the
+    // epilogue warps grow to 216 (128 x 120 released, 256 x 48 taken).
     if (warp == 0) {
-        // ---- producer + MMA issue: the whole warp runs the loop (a lone lane of a diverged warp runs
-        // slowly), lane 0 issues ----------------------------------------------------------------------
-        const uint32_t qbar = smem_u32(&bars.q_full);
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        // ---- producer: the whole warp runs the loop (a lone lane of a diverged warp runs slowly), lane 0 copies ----
         const int n_q_tiles = p.n_cols > 128 ? 2 : 1;
-        const int row0 = (((p.layer0 + l) * p.batch + b) * p.Hkv + h) * p.max_blocks;
-        auto load_tile = [&](int i) {  // lane 0 only
-            const int slot = i % stages;
-            const uint32_t full = smem_u32(&bars.sum_full[slot]);
-            mbar_expect_tx(full, 2 * kSumTileBytes);
-            const uint32_t dst = sum_smem + slot * 2 * kSumTileBytes;
-            const int row = row0 + (tile_begin + i) * kTileBlocks;
-            for (int half = 0; half < 2; ++half) {
-                tma_load_2d(dst + half * 16384, &p.tm_kmax, half * 64, row, full);
-                tma_load_2d(dst + kSumTileBytes + half * 16384, &p.tm_kmin, half * 64, row, full);
+        ScoreIter it;
+        it.init(p);
+        ScoreSeg s;
+        uint32_t g = 0;  // tiles so far, across stretches
+        bool ok = true;
+        for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+            // Q may only be replaced once the contractions of the previous stretch have read it
+            if (sidx > 0) ok &= mbar_wait(smem_u32(&bars.q_empty), (sidx - 1) & 1, abort_flag, p.workspace, 27);
+            if (lane == 0 && ok) {
+                const uint32_t qbar = smem_u32(&bars.q_full);
+                mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
+                for (int t = 0; t < n_q_tiles; ++t)
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_3d(q_smem + half * 32768 + t * 16384, &p.tm_q, half * 64, s.h * p.G,
+                                    s.lb * p.M_max + p.tok0 + t * tok_per_tile, qbar);
             }
-        };
-        if (lane == 0) {
-            mbar_expect_tx(qbar, (uint32_t)(n_q_tiles * 32768));
-            for (int t = 0; t < n_q_tiles; ++t)
-                for (int half = 0; half < 2; ++half)
-                    tma_load_3d(q_smem + half * 32768 + t * 16384, &p.tm_q, half * 64, h * p.G,
-                                lb * p.M_max + p.tok0 + t * tok_per_tile, qbar);
-            load_tile(0);
+            __syncwarp();
+            const int row0 = (((p.layer0 + s.l) * p.batch + s.b) * p.Hkv + s.h) * p.max_blocks;
+            for (int t = s.t0; t < s.t1 && ok; ++t, ++g) {
+                for (uint32_t which = 0; which < 2; ++which) {  // the Kmax rows of the tile, then its Kmin rows
+                    const uint32_t u = 2 * g + which, slot = u % stages;
+                    if (u >= (uint32_t)stages)
+                        ok &= mbar_wait(smem_u32(&bars.sum_empty[slot]), ((u / stages) - 1) & 1, abort_flag, p.workspace, 21);
+                    if (lane == 0 && ok) {
+                        const uint32_t full = smem_u32(&bars.sum_full[slot]);
+                        mbar_expect_tx(full, kSumTileBytes);
+                        const uint32_t dst = sum_smem + slot * kSumTileBytes;
+                        const int row = row0 + t * kTileBlocks;
+                        for (int half = 0; half < 2; ++half)
+                            tma_load_2d(dst + half * 16384, which ? &p.tm_kmin : &p.tm_kmax, half * 64, row, full);
+                    }
+                    __syncwarp();
+                }
+            }
         }
-        __syncwarp();
+    } else if (warp == 1 || warp == 2) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        // ---- MMA issue: warp 1 issues Kmax . Q into region 0, warp 2 Kmin . Q into region 1.  The whole warp runs the
+        // loop, lane 0 issues.  A thread that issues also waits and commits, and the tensor pipe queues next to
+        // nothing ahead, so the barrier work of one warp overlaps the contractions of the other.
+        // A warp meets every other use of a ring slot (five slots, uses alternate between Kmax and Kmin), so it
+        // waits on the same parity each time; that is sound because the use in between has completed by then: a warp
+        // can issue tile g - 1 only after the epilogue has reached tile g - 2, hence after the other warp's
+        // contractions of tile g - 3, whose slot use is the one in between.
+        // Channel-wise form: one accumulator per tile, so warp 1 issues every tile, alternating between the regions
+        // (a warp that took every other tile would skip ring-slot phases without that guarantee); warp 2 only
+        // takes part in releasing Q.
         // descriptors: constant upper word (8-row group stride 1024 B, version, 128-byte swizzle); lower word =
         // 16-byte address, leading offset 16 B
+        const uint32_t w = (uint32_t)(warp - 1);
         const uint32_t desc_hi = (uint32_t)((1024u >> 4) | (1u << 14) | (2u << 29));
         const uint32_t q_lo = ((q_smem >> 4) & 0x3FFFu) | (1u << 16);
         const uint32_t sum_lo = ((sum_smem >> 4) & 0x3FFFu) | (1u << 16);
         const uint32_t qneg_lo = ((qneg_smem >> 4) & 0x3FFFu) | (1u << 16);
-        bool ok = mbar_wait(qbar, 0, abort_flag, p.workspace, 20);
-        if (kCw) ok &= mbar_wait(smem_u32(&bars.q_split), 0, abort_flag, p.workspace, 25);
-        for (int i = 0; i < n_tiles; ++i) {
-            if (stages > 1 && i + 1 < n_tiles) {  // the next tile goes into the other stage while this one is used
-                const int use = i + 1;
-                if (use >= stages)
-                    ok &= mbar_wait(smem_u32(&bars.sum_empty[use % stages]), ((use / stages) - 1) & 1,
-                                    abort_flag, p.workspace, 21);
-                if (lane == 0 && ok) load_tile(use);
-                __syncwarp();
-            }
-            const int slot = i % stages;
-            ok &= mbar_wait(smem_u32(&bars.sum_full[slot]), (i / stages) & 1, abort_flag, p.workspace, 22);
-            if (i > 0) ok &= mbar_wait(smem_u32(&bars.d_empty), (i - 1) & 1, abort_flag, p.workspace, 23);
-            if (!ok) break;  // a wait gave up: nothing more is copied or issued
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t a_max = sum_lo + (uint32_t)slot * (2 * kSumTileBytes >> 4), a_min = a_max + (kSumTileBytes >> 4);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t a_off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
-                    const uint32_t b_off = (uint32_t)((kk >> 2) * 32768 + (kk & 3) * 32) >> 4;
-                    const uint64_t bdesc = ((uint64_t)desc_hi << 32) | (q_lo + b_off);
-                    mma_ss(tmem, ((uint64_t)desc_hi << 32) | (a_max + a_off), bdesc, idesc, kk > 0);
-                    // channel-wise: Kmin . q- joins Kmax . q+ in the same accumulator
-                    if (kCw)
-                        mma_ss(tmem, ((uint64_t)desc_hi << 32) | (a_min + a_off), ((uint64_t)desc_hi << 32) | (qneg_lo + b_off),
-                               idesc, 1);
-                    else
-                        mma_ss(tmem + 256, ((uint64_t)desc_hi << 32) | (a_min + a_off), bdesc, idesc, kk > 0);
-                }
-                tc_commit(smem_u32(&bars.d_full));
-                tc_commit(smem_u32(&bars.sum_empty[slot]));
-            }
-            __syncwarp();
-            if (stages == 1 && i + 1 < n_tiles) {
-                // a single stage: the next tile can only follow the contractions just issued (their completion is
-                // release number i of the stage); it still overlaps this tile's reduction
-                ok &= mbar_wait(smem_u32(&bars.sum_empty[0]), i & 1, abort_flag, p.workspace, 21);
-                if (lane == 0 && ok) load_tile(i + 1);
-                __syncwarp();
-            }
-        }
-        (void)ok;
-    } else if (warp >= 2) {
-        // ---- epilogue: thread <-> block of the tile -----------------------------------------------
-        const int q = warp & 3;  // tensor-memory lane quarter of this warp
-        const int blk_in_tile = q * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const uint32_t idesc = make_idesc((uint32_t)p.n_cols, false);
+
+        ScoreIter it;
+        it.init(p);
+        ScoreSeg s;
+        uint32_t g = 0;  // tiles so far, across stretches
         bool ok = true;
-        if (kCw) {
-            // split Q by sign in place: q+ stays where Q landed, q- goes to the buffer behind it (same swizzled layout,
-            // the split is element-wise).  A bfloat16 is negative when its top bit is set.
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, p.workspace, 26));
-            uint4* qp = reinterpret_cast<uint4*>(smem);
-            uint4* qn = reinterpret_cast<uint4*>(smem + kScoreQBytes);
-            for (int v = threadIdx.x - 64; v < kScoreQBytes / 16; v += 128) {
-                const uint4 w = qp[v];
-                const uint32_t in[4] = {w.x, w.y, w.z, w.w};
-                uint32_t pos[4], neg[4];
+        for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+            ok &= mbar_wait(smem_u32(&bars.q_full), sidx & 1, abort_flag, p.workspace, 20);
+            if (kCw) ok &= mbar_wait(smem_u32(&bars.q_split), sidx & 1, abort_flag, p.workspace, 25);
+            for (int t = s.t0; t < s.t1; ++t, ++g) {
+                if (!kCw || w == 0) {
+                    const uint32_t r = kCw ? (g & 1u) : w;    // accumulator region of this tile
+                    const uint32_t use = kCw ? (g >> 1) : g;  // earlier uses of that region
+                    const uint32_t d = tmem + r * 256u;
+                    const uint32_t rfull = smem_u32(&bars.r_full[r]), rempty = smem_u32(&bars.r_empty[r]);
+                    const uint32_t u0 = kCw ? 2 * g : 2 * g + w, s0 = u0 % stages;
+                    const uint32_t u1 = 2 * g + 1, s1 = u1 % stages;  // channel-wise only: the tile's Kmin rows
+                    ok &= mbar_wait(smem_u32(&bars.sum_full[s0]), (u0 / stages) & 1, abort_flag, p.workspace, 22);
+                    if (kCw) ok &= mbar_wait(smem_u32(&bars.sum_full[s1]), (u1 / stages) & 1, abort_flag, p.workspace, 22);
+                    if (use > 0) ok &= mbar_wait(rempty, (use - 1) & 1, abort_flag, p.workspace, 23);
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a0 = sum_lo + s0 * (kSumTileBytes >> 4), a1 = sum_lo + s1 * (kSumTileBytes >> 4);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t m = ((in[e] >> 15) & 0x00010001u) * 0xFFFFu;  // all ones in the negative halves
-                    neg[e] = in[e] & m;
-                    pos[e] = in[e] & ~m;
-                }
-                qp[v] = make_uint4(pos[0], pos[1], pos[2], pos[3]);
-                qn[v] = make_uint4(neg[0], neg[1], neg[2], neg[3]);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor pipe reads these through the async proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.q_split));
-        }
-        for (int i = 0; i < n_tiles && ok; ++i) {
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full), i & 1, abort_flag, p.workspace, 24));
-            if (!ok) break;
-            tc_fence_after();
-            // four independent partial reductions: a single chain through one register would leave this
-            // warp, alone on its scheduler, waiting out the latency of every instruction
-            const bool is_max = p.reduce == SPECPV_REDUCE_MAX;
-            float r4[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) r4[e] = is_max ? -INFINITY : 0.f;
-            for (int c0 = (col_begin / 64) * 64; c0 < col_end; c0 += 64) {
-                uint32_t vmax[64], vmin[64];
-                TMEM_LD32(tmem + lane_addr + c0, vmax);
-                TMEM_LD32(tmem + lane_addr + c0 + 32, (vmax + 32));
-                if (!kCw) {
-                    TMEM_LD32(tmem + lane_addr + 256 + c0, vmin);
-                    TMEM_LD32(tmem + lane_addr + 256 + c0 + 32, (vmin + 32));
-                }
-                tmem_wait_ld();
-                if (kCw) {  // one accumulator already holds the score: max(x, x) = x below
-#pragma unroll
-                    for (int k = 0; k < 64; ++k) vmin[k] = vmax[k];
-                }
-                const bool whole = c0 >= col_begin && c0 + 64 <= col_end;  // warp-uniform
-                if (whole && !is_max) {
-#pragma unroll
-                    for (int k = 0; k < 64; ++k)
-                        r4[k & 3] += fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
-                } else if (whole) {
-#pragma unroll
-                    for (int k = 0; k < 64; ++k)
-                        r4[k & 3] = fmax3(r4[k & 3], __uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 64; ++k) {
-                        const int c = c0 + k;
-                        const float sc = fmaxf(__uint_as_float(vmax[k]), __uint_as_float(vmin[k]));
-                        if (c >= col_begin && c < col_end) r4[k & 3] = is_max ? fmaxf(r4[k & 3], sc) : r4[k & 3] + sc;
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t a_off = (uint32_t)((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                            const uint32_t b_off = (uint32_t)((kk >> 2) * 32768 + (kk & 3) * 32) >> 4;
+                            mma_ss(d, ((uint64_t)desc_hi << 32) | (a0 + a_off), ((uint64_t)desc_hi << 32) | (q_lo + b_off), idesc, kk > 0);
+                            // channel-wise: Kmin . q- joins Kmax . q+ in the same accumulator
+                            if (kCw)
+                                mma_ss(d, ((uint64_t)desc_hi << 32) | (a1 + a_off), ((uint64_t)desc_hi << 32) | (qneg_lo + b_off), idesc, 1);
+                        }
+                        tc_commit(rfull);
+                        tc_commit(smem_u32(&bars.sum_empty[s0]));
+                        if (kCw) tc_commit(smem_u32(&bars.sum_empty[s1]));
                     }
                 }
+                // Q is released by both warps: each commit covers the contractions its own thread has issued
+                if (t == s.t1 - 1 && lane == 0) tc_commit(smem_u32(&bars.q_empty));
+                __syncwarp();
+                if (!ok) break;  // a wait gave up: nothing is issued past this tile
             }
-            float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty));
-            const int blk = (tile_begin + i) * kTileBlocks + blk_in_tile;
-            if (blk < nb) {
-                float* dst = p.scores + ((size_t)lb * p.Hkv + h) * p.max_blocks + blk;
-                if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)denom;
-                if (combine) red = is_max ? fmaxf(red, *dst) : red + *dst;
-                *dst = red;
+        }
+    } else if (warp == 3) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        // ---- epilogue: thread <-> (block of the tile, half of the query rows) ------------------------------------
+        const int q = warp & 3;           // tensor-memory lane quarter of this warp
+        const int ch = (warp - 4) >> 2;   // its half of the query rows: accumulator columns [ch * 128, ch * 128 + 128)
+        const int blk_in_tile = q * 32 + lane;
+        const uint32_t my_cols = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 128);
+        const bool is_max = p.reduce == SPECPV_REDUCE_MAX;
+        const bool combine = p.accumulate && p.reduce != SPECPV_REDUCE_LAST;
+        ScoreIter it;
+        it.init(p);
+        ScoreSeg s;
+        uint32_t g = 0;
+        bool ok = true;
+        for (int sidx = 0; ok && it.next(p, s); ++sidx) {
+            if (kCw) {
+                // split Q by sign in place: q+ stays where Q landed, q- goes to the buffer behind it (same swizzled layout,
+                // the split is element-wise).  A bfloat16 is negative when its top bit is set.
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full), sidx & 1, abort_flag, p.workspace, 26));
+                if (!ok) break;
+                uint4* qp = reinterpret_cast<uint4*>(smem);
+                uint4* qn = reinterpret_cast<uint4*>(smem + kScoreQBytes);
+                for (int v = threadIdx.x - 128; v < kScoreQBytes / 16; v += 256) {
+                    const uint4 w = qp[v];
+                    const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+                    uint32_t pos[4], neg[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t m = ((in[e] >> 15) & 0x00010001u) * 0xFFFFu;  // all ones in the negative halves
+                        neg[e] = in[e] & m;
+                        pos[e] = in[e] & ~m;
+                    }
+                    qp[v] = make_uint4(pos[0], pos[1], pos[2], pos[3]);
+                    qn[v] = make_uint4(neg[0], neg[1], neg[2], neg[3]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor pipe reads these through the async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.q_split));
+            }
+            // the rows of this thread's half that count: columns [lo, hi) of its 128
+            const int lo = max(s.col_begin - ch * 128, 0), hi = min(s.col_end - ch * 128, 128);
+            for (int t = s.t0; t < s.t1 && ok; ++t, ++g) {
+                // four independent partial reductions: a single chain through one register would leave the warp
+                // waiting out the latency of every instruction
+                float r4[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) r4[e] = is_max ? -INFINITY : 0.f;
+                // one 32-column chunk of scores sc[k] = column c0 + k of this thread's half
+                auto reduce_chunk = [&](int c0, const float* sc) {
+                    if (c0 >= lo && c0 + 32 <= hi) {  // warp-uniform
+                        if (!is_max) {
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) r4[k & 3] += sc[k];
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) r4[k & 3] = fmaxf(r4[k & 3], sc[k]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            if (c0 + k >= lo && c0 + k < hi) r4[k & 3] = is_max ? fmaxf(r4[k & 3], sc[k]) : r4[k & 3] + sc[k];
+                    }
+                };
+                if (!kCw) {
+                    // Dmax of this half into registers, and its region is free for the next tile at once
+                    uint32_t hold[128];
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[0]), g & 1, abort_flag, p.workspace, 24));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lo < hi) {
+                        TMEM_LD32(my_cols, hold);
+                        TMEM_LD32(my_cols + 32, (hold + 32));
+                        TMEM_LD32(my_cols + 64, (hold + 64));
+                        TMEM_LD32(my_cols + 96, (hold + 96));
+                        tmem_wait_ld();
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[0]));
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[1]), g & 1, abort_flag, p.workspace, 24));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lo < hi) {
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            if (c4 * 32 + 32 <= lo || c4 * 32 >= hi) continue;  // warp-uniform
+                            uint32_t v[32];
+                            TMEM_LD32(my_cols + 256 + c4 * 32, v);
+                            tmem_wait_ld();
+                            float sc[32];
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) sc[k] = fmaxf(__uint_as_float(hold[c4 * 32 + k]), __uint_as_float(v[k]));
+                            reduce_chunk(c4 * 32, sc);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[1]));
+                } else {
+                    // one accumulator holds the score; the tiles alternate between the regions
+                    const uint32_t r = g & 1u;
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[r]), (g >> 1) & 1, abort_flag, p.workspace, 24));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lo < hi) {
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            if (c4 * 32 + 32 <= lo || c4 * 32 >= hi) continue;  // warp-uniform
+                            uint32_t v[32];
+                            TMEM_LD32(my_cols + r * 256u + c4 * 32, v);
+                            tmem_wait_ld();
+                            float sc[32];
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) sc[k] = __uint_as_float(v[k]);
+                            reduce_chunk(c4 * 32, sc);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    // the warps of the lower half release the region only after the exchange below: the next use of
+                    // this region is tile g + 2, whose exchange reuses this tile's slot
+                    if (lane == 0 && ch == 1) mbar_arrive(smem_u32(&bars.r_empty[r]));
+                }
+                float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
+                // The two halves of the query rows meet in shared memory.  The slot of tile g is free again by tile
+                // g + 2: the contractions of tile g + 2 wait for every epilogue warp to have released a region after
+                // its exchange of tile g (region 0 of tile g + 1, or in the channel-wise form the region of tile g itself).
+                if (ch == 1) {
+                    xch[g & 1][blk_in_tile] = red;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.x_full[g & 1]));
+                } else {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.x_full[g & 1]), (g >> 1) & 1, abort_flag, p.workspace, 28));
+                    if (!ok) break;
+                    const float other = xch[g & 1][blk_in_tile];
+                    if (kCw) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[g & 1]));
+                    }
+                    red = is_max ? fmaxf(red, other) : red + other;
+                    const int blk = t * kTileBlocks + blk_in_tile;
+                    if (blk < s.nb) {
+                        float* dst = p.scores + ((size_t)s.lb * p.Hkv + s.h) * p.max_blocks + blk;
+                        if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)s.denom;
+                        if (combine) red = is_max ? fmaxf(red, *dst) : red + *dst;
+                        *dst = red;
+                    }
+                }
             }
         }
     }
@@ -325,15 +463,11 @@ specpv_status launch_scores_tc(const ScoreParams& sp, int n_layers_call, int n_l
     p.workspace = sp.workspace;
     p.layer0 = sp.layer0; p.batch = sp.batch; p.M_max = sp.M_max; p.Hkv = sp.Hkv; p.G = sp.G; p.bs = sp.bs;
     p.max_blocks = sp.max_blocks; p.reduce = sp.reduce;
-    const int n_tiles = (max_nb + kTileBlocks - 1) / kTileBlocks;
-    const int heads = sp.Hkv * n_layers_call * sp.batch;
-    // enough CTAs to fill the machine, but at least a few tiles each so that Q is amortised
-    int ctas_x = (2 * 148 + heads - 1) / heads;
-    if (ctas_x > n_tiles) ctas_x = n_tiles;
-    if (ctas_x < 1) ctas_x = 1;
-    p.tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
-    ctas_x = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
-    dim3 grid(ctas_x, sp.Hkv, n_layers_call * sp.batch);
+    // one CTA per SM, each with an equal share of all tile positions; fewer CTAs when there are fewer tiles than SMs
+    p.tiles_max = (max_nb + kTileBlocks - 1) / kTileBlocks;
+    p.n_heads = sp.Hkv * n_layers_call * sp.batch;
+    const long long total = (long long)p.n_heads * p.tiles_max;
+    dim3 grid((unsigned)(total < kScoreCtas ? total : kScoreCtas), 1, 1);
     // The accumulator holds 256 query rows; a step with more (the chain and the tree of a refresh) goes through in
     // passes over the step's tokens, each later pass combining with what is there (sum of per-pass means, or max).
     const int tok_per_pass = 256 / sp.G;
