@@ -39,7 +39,7 @@ ACCEPT_LEN = 4  # tokens committed per step: the paper's mean accept length is 3
 
 # DRAM bytes (read + write) of one full-verification attention launch per layer, from the ncu capture of the
 # 2-layer case summarised in profiles/attn_tc_kernel_llama_128k.md; the traffic is proportional to the layers streamed.
-NCU_DRAM_BYTES_PER_LAYER = {"llama_128k": (1.075295e9 + 5.69728e6) / 2}
+NCU_DRAM_BYTES_PER_LAYER = {"llama_128k": (1.075296e9 + 5.433088e6) / 2}
 
 
 def ncu_traffic_bytes(workload: str, n_layers: int):
