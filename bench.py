@@ -455,7 +455,7 @@ def offloaded_refresh(st, layers=4, iters=3):
 def score_variants(st, peaks, iters=10):
     """Block scoring and selection in their variants (Eq. 3's reductions mean / max / last, Eq. 2 as printed and in
     its channel-wise form, selection per head and shared by the heads), each call alone over all layers.  Scoring
-    reads the summaries once: `frac` is against the HBM time of those bytes."""
+    reads the summaries once: `frac` is against the HBM time of those bytes.  Measured after a one-second pause."""
     B, w, L, M, batch = st["B"], st["w"], st["L"], st["M"], st["batch"]
     c = w.cfg
     Hq, Hkv, d, bs = c["Hq"], c["Hkv"], c["d"], c["bs"]
@@ -475,6 +475,10 @@ def score_variants(st, peaks, iters=10):
             b.record()
         torch.cuda.synchronize(dev)
         return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+    # these are kernel-alone figures (compared with the burst copy rate): let the device settle after the heavy sections
+    # that ran before, which leave it at a power-limited clock for a while
+    torch.cuda.synchronize(dev)
+    time.sleep(1.0)
     scores = torch.zeros_like(st["scores"])
     idx = torch.zeros_like(st["idx"])
     count = torch.zeros_like(st["count"])

@@ -15,13 +15,14 @@
 // into another head.  Tensor memory holds two accumulator regions of 256 columns (one per query row): Dmax in the
 // first, Dmin in the second.  Each product has its own issuing warp and its own stream of ring slots, so the barrier
 // work of one overlaps the contractions of the other, and a region is free again as soon as the epilogue has READ it:
-// Dmax is read into registers while the Dmin contractions run, the next tile's Dmax contractions run while the
-// epilogue takes max(Dmax, Dmin) and reduces.  The tensor pipe never waits for the reduction.  (The channel-wise form
-// has one accumulator per tile, so its tiles simply alternate between the two regions and the two issuing warps.)
+// Dmax is read into registers while the Dmin contractions run; Dmin is read in two round trips, only the maximum is
+// taken, and its region is released before the reduction over the rows; the next tile's contractions run meanwhile.
+// (The channel-wise form has one accumulator per tile: its tiles alternate between the two regions, issued by one warp.)
 //   warp 0      TMA producer: Q of a head, then per tile its Kmax rows and its Kmin rows through a ring of 32 KB slots
 //   warps 1, 2  MMA issue: Dmax / Dmin (warp 1 also allocates the tensor memory)
 //   warps 4-11  epilogue: thread <-> block of the tile (tensor-memory lane) and one half of the query rows; reduces
-//               over its rows (mean, max, or the rows of the "last" query); the two halves meet in shared memory
+//               over its rows (mean, max, or the rows of the "last" query); the two halves meet in shared memory, the
+//               lower half picking the upper half's result up one tile later
 // Every wait is bounded; after a wait that gave up the loops end and nothing more is copied or issued.
 #include "aux_kernels.cuh"
 #include "tc_common.cuh"
@@ -64,7 +65,7 @@ struct __align__(8) ScoreBarriers {
     uint64_t sum_empty[kScoreStages];
     uint64_t r_full[2];                // per accumulator region: the contractions of a tile are complete
     uint64_t r_empty[2];               // ... and the eight epilogue warps have read the region
-    uint64_t x_full[2];                // the warps of the upper half of the query rows have left their partial results (tile parity)
+    uint64_t x_full[3];                // the warps of the upper half of the query rows have left their partial results (tile mod 3)
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -125,7 +126,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ ScoreBarriers bars;
-    __shared__ float xch[2][kTileBlocks];  // partial results of the upper half of the query rows, by tile parity
+    __shared__ float xch[3][kTileBlocks];  // partial results of the upper half of the query rows, by tile mod 3
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const uint32_t q_smem = smem_u32(smem);
@@ -146,8 +147,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         for (int r = 0; r < 2; ++r) {
             mbar_init(smem_u32(&bars.r_full[r]), 1);
             mbar_init(smem_u32(&bars.r_empty[r]), 8);
-            mbar_init(smem_u32(&bars.x_full[r]), 4);
         }
+        for (int x = 0; x < 3; ++x) mbar_init(smem_u32(&bars.x_full[x]), 4);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     const int tok_per_tile = 128 / p.G;
 
     // Register budget: 384 threads start with 168 registers each; the control warps keep 48, which is what lets the
-    // epilogue warps grow to 216 (128 x 120 released, 256 x 48 taken).
+    // epilogue warps grow to 224 (128 x 120 released, 256 x 56 taken).
     if (warp == 0) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         // ---- producer: the whole warp runs the loop (a lone lane of a diverged warp runs slowly), lane 0 copies ----
@@ -270,7 +271,7 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
     } else if (warp == 3) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // ---- epilogue: thread <-> (block of the tile, half of the query rows) ------------------------------------
         const int q = warp & 3;           // tensor-memory lane quarter of this warp
         const int ch = (warp - 4) >> 2;   // its half of the query rows: accumulator columns [ch * 128, ch * 128 + 128)
@@ -283,6 +284,24 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
         ScoreSeg s;
         uint32_t g = 0;
         bool ok = true;
+        // lower half: the tile whose exchange with the upper half is still to come
+        bool have_prev = false;
+        float prev_red = 0.f, prev_denom = 1.f;
+        uint32_t xs = 0, xp = 0, prev_xs = 0, prev_xp = 0;  // exchange slot (tile mod 3) and its parity, now and of the pending tile
+        float* prev_dst = nullptr;
+        auto finish_prev = [&]() -> bool {
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.x_full[prev_xs]), prev_xp, abort_flag, p.workspace, 28)))
+                return false;
+            float red = xch[prev_xs][blk_in_tile];
+            red = is_max ? fmaxf(prev_red, red) : prev_red + red;
+            if (prev_dst) {
+                if (p.reduce != SPECPV_REDUCE_MAX) red /= prev_denom;
+                if (combine) red = is_max ? fmaxf(red, *prev_dst) : red + *prev_dst;
+                *prev_dst = red;
+            }
+            have_prev = false;
+            return true;
+        };
         for (int sidx = 0; ok && it.next(p, s); ++sidx) {
             if (kCw) {
                 // split Q by sign in place: q+ stays where Q landed, q- goes to the buffer behind it (same swizzled layout,
@@ -318,7 +337,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                 for (int e = 0; e < 4; ++e) r4[e] = is_max ? -INFINITY : 0.f;
                 // one 32-column chunk of scores sc[k] = column c0 + k of this thread's half
                 auto reduce_chunk = [&](int c0, const float* sc) {
-                    if (c0 >= lo && c0 + 32 <= hi) {  // warp-uniform
+                    if (c0 + 32 <= lo || c0 >= hi) return;  // warp-uniform
+                    if (c0 >= lo && c0 + 32 <= hi) {
                         if (!is_max) {
 #pragma unroll
                             for (int k = 0; k < 32; ++k) r4[k & 3] += sc[k];
@@ -330,6 +350,21 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
                             if (c0 + k >= lo && c0 + k < hi) r4[k & 3] = is_max ? fmaxf(r4[k & 3], sc[k]) : r4[k & 3] + sc[k];
+                    }
+                };
+                // Channel-wise form: the 128 columns of a region in four chunks, the load of chunk c + 1 in flight while
+                // chunk c is reduced (tcgen05.wait::ld waits for every load issued so far, so it comes after the arithmetic).
+                auto reduce_region = [&](uint32_t cols) {
+                    uint32_t va[32], vb[32];
+                    TMEM_LD32(cols, va);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t* cur = (c4 & 1) ? vb : va;
+                        uint32_t* nxt = (c4 & 1) ? va : vb;
+                        if (c4 < 3) TMEM_LD32(cols + (c4 + 1) * 32, nxt);
+                        reduce_chunk(c4 * 32, reinterpret_cast<const float*>(cur));
+                        if (c4 < 3) tmem_wait_ld();
                     }
                 };
                 if (!kCw) {
@@ -348,77 +383,75 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[0]));
+                    // while the Dmin contractions of this tile run: the lower half finishes the previous tile
+                    if (ch == 0 && have_prev) {
+                        ok = finish_prev();
+                        if (!ok) break;
+                    }
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[1]), g & 1, abort_flag, p.workspace, 24));
                     if (!ok) break;
                     tc_fence_after();
+                    // Dmin in two round trips of 64 columns (a round trip to tensor memory costs about 300 cycles while the
+                    // tensor pipe is writing the other region, whatever it carries); only the maximum is taken before the
+                    // region is released, the reduction over the rows follows from registers
                     if (lo < hi) {
 #pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            if (c4 * 32 + 32 <= lo || c4 * 32 >= hi) continue;  // warp-uniform
-                            uint32_t v[32];
-                            TMEM_LD32(my_cols + 256 + c4 * 32, v);
+                        for (int c2 = 0; c2 < 2; ++c2) {
+                            if (c2 * 64 + 64 <= lo || c2 * 64 >= hi) continue;  // warp-uniform
+                            uint32_t v[64];
+                            TMEM_LD32(my_cols + 256 + c2 * 64, v);
+                            TMEM_LD32(my_cols + 256 + c2 * 64 + 32, (v + 32));
                             tmem_wait_ld();
-                            float sc[32];
 #pragma unroll
-                            for (int k = 0; k < 32; ++k) sc[k] = fmaxf(__uint_as_float(hold[c4 * 32 + k]), __uint_as_float(v[k]));
-                            reduce_chunk(c4 * 32, sc);
+                            for (int k = 0; k < 64; ++k)
+                                hold[c2 * 64 + k] = __float_as_uint(fmaxf(__uint_as_float(hold[c2 * 64 + k]), __uint_as_float(v[k])));
                         }
                     }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[1]));
+                    if (lo < hi) {
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) reduce_chunk(c4 * 32, reinterpret_cast<const float*>(hold + c4 * 32));
+                    }
                 } else {
                     // one accumulator holds the score; the tiles alternate between the regions
                     const uint32_t r = g & 1u;
+                    if (ch == 0 && have_prev) {
+                        ok = finish_prev();
+                        if (!ok) break;
+                    }
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[r]), (g >> 1) & 1, abort_flag, p.workspace, 24));
                     if (!ok) break;
                     tc_fence_after();
-                    if (lo < hi) {
-#pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            if (c4 * 32 + 32 <= lo || c4 * 32 >= hi) continue;  // warp-uniform
-                            uint32_t v[32];
-                            TMEM_LD32(my_cols + r * 256u + c4 * 32, v);
-                            tmem_wait_ld();
-                            float sc[32];
-#pragma unroll
-                            for (int k = 0; k < 32; ++k) sc[k] = __uint_as_float(v[k]);
-                            reduce_chunk(c4 * 32, sc);
-                        }
-                    }
+                    if (lo < hi) reduce_region(my_cols + r * 256u);
                     tc_fence_before();
                     __syncwarp();
-                    // the warps of the lower half release the region only after the exchange below: the next use of
-                    // this region is tile g + 2, whose exchange reuses this tile's slot
-                    if (lane == 0 && ch == 1) mbar_arrive(smem_u32(&bars.r_empty[r]));
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[r]));
                 }
-                float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
-                // The two halves of the query rows meet in shared memory.  The slot of tile g is free again by tile
-                // g + 2: the contractions of tile g + 2 wait for every epilogue warp to have released a region after
-                // its exchange of tile g (region 0 of tile g + 1, or in the channel-wise form the region of tile g itself).
+                const float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
+                // The two halves of the query rows meet in shared memory, in one of three slots (tile mod 3).  The upper half
+                // leaves its partial result; the lower half keeps its own and picks the other up one tile later, so that it
+                // never waits for the upper half inside a tile.  The slot of tile g is rewritten at tile g + 3, whose
+                // contractions cannot start before every warp has released a region of tile g + 2 (Dmax) or g + 1
+                // (channel-wise form), which the lower half does after its exchange of tile g.
                 if (ch == 1) {
-                    xch[g & 1][blk_in_tile] = red;
+                    xch[xs][blk_in_tile] = red;
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars.x_full[g & 1]));
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.x_full[xs]));
                 } else {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.x_full[g & 1]), (g >> 1) & 1, abort_flag, p.workspace, 28));
-                    if (!ok) break;
-                    const float other = xch[g & 1][blk_in_tile];
-                    if (kCw) {
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[g & 1]));
-                    }
-                    red = is_max ? fmaxf(red, other) : red + other;
                     const int blk = t * kTileBlocks + blk_in_tile;
-                    if (blk < s.nb) {
-                        float* dst = p.scores + ((size_t)s.lb * p.Hkv + s.h) * p.max_blocks + blk;
-                        if (p.reduce != SPECPV_REDUCE_MAX) red /= (float)s.denom;
-                        if (combine) red = is_max ? fmaxf(red, *dst) : red + *dst;
-                        *dst = red;
-                    }
+                    prev_red = red;
+                    prev_xs = xs;
+                    prev_xp = xp;
+                    prev_denom = (float)s.denom;
+                    prev_dst = blk < s.nb ? p.scores + ((size_t)s.lb * p.Hkv + s.h) * p.max_blocks + blk : nullptr;
+                    have_prev = true;
                 }
+                if (++xs == 3) { xs = 0; xp ^= 1; }
             }
         }
+        if (ok && ch == 0 && have_prev) ok = finish_prev();
     }
     tc_fence_before();
     __syncthreads();
