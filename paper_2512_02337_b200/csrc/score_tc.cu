@@ -352,21 +352,6 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                             if (c0 + k >= lo && c0 + k < hi) r4[k & 3] = is_max ? fmaxf(r4[k & 3], sc[k]) : r4[k & 3] + sc[k];
                     }
                 };
-                // Channel-wise form: the 128 columns of a region in four chunks, the load of chunk c + 1 in flight while
-                // chunk c is reduced (tcgen05.wait::ld waits for every load issued so far, so it comes after the arithmetic).
-                auto reduce_region = [&](uint32_t cols) {
-                    uint32_t va[32], vb[32];
-                    TMEM_LD32(cols, va);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint32_t* cur = (c4 & 1) ? vb : va;
-                        uint32_t* nxt = (c4 & 1) ? va : vb;
-                        if (c4 < 3) TMEM_LD32(cols + (c4 + 1) * 32, nxt);
-                        reduce_chunk(c4 * 32, reinterpret_cast<const float*>(cur));
-                        if (c4 < 3) tmem_wait_ld();
-                    }
-                };
                 if (!kCw) {
                     // Dmax of this half into registers, and its region is free for the next tile at once
                     uint32_t hold[128];
@@ -424,10 +409,22 @@ __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __gri
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.r_full[r]), (g >> 1) & 1, abort_flag, p.workspace, 24));
                     if (!ok) break;
                     tc_fence_after();
-                    if (lo < hi) reduce_region(my_cols + r * 256u);
+                    // the whole half in one round trip to tensor memory, the region released before the reduction
+                    uint32_t v[128];
+                    if (lo < hi) {
+                        TMEM_LD32(my_cols + r * 256u, v);
+                        TMEM_LD32(my_cols + r * 256u + 32, (v + 32));
+                        TMEM_LD32(my_cols + r * 256u + 64, (v + 64));
+                        TMEM_LD32(my_cols + r * 256u + 96, (v + 96));
+                        tmem_wait_ld();
+                    }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars.r_empty[r]));
+                    if (lo < hi) {
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) reduce_chunk(c4 * 32, reinterpret_cast<const float*>(v + c4 * 32));
+                    }
                 }
                 const float red = is_max ? fmaxf(fmaxf(r4[0], r4[1]), fmaxf(r4[2], r4[3])) : (r4[0] + r4[1]) + (r4[2] + r4[3]);
                 // The two halves of the query rows meet in shared memory, in one of three slots (tile mod 3).  The upper half
