@@ -120,6 +120,9 @@ struct ScoreIter {
     }
 };
 
+// dynamic + static shared memory of the kernel below must fit the 227 KB a CTA may have
+static_assert(kScoreSmem + sizeof(ScoreBarriers) + 3 * kTileBlocks * sizeof(float) + 64 <= 227 * 1024, "shared memory of scores_tc_kernel");
+
 // kCw: the channel-wise form (a compile-time switch).
 template <bool kCw>
 __global__ void __launch_bounds__(kScoreThreads, 1) scores_tc_kernel(const __grid_constant__ ScoreTcParams p) {
