@@ -651,7 +651,11 @@ def main():
     c = st["w"].cfg
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local_rank)
     sampler.start()
-    time.sleep(0.3)  # let the sampler deliver its first rows before the warm-up starts
+    # Generating 17 GB of synthetic caches leaves the device warm and at a power-limited clock for a while: let it settle,
+    # so that the warm-up and the timed steps start from the same state on every run (the sampler also delivers its first
+    # rows meanwhile).
+    torch.cuda.synchronize(dev)
+    time.sleep(2.0)
     ms_step, full_ms, part_ms, launches, window = timed_loop(st, args.steps, warmup, False, barrier)
     clocks = sampler.stop(*window)
     e2e = None
@@ -713,6 +717,7 @@ def main():
                    "step": "refresh step (full verify + commit + scores + select + gather) + partial step "
                            "(partial verify + commit)",
                    "l2": "inputs larger than L2 (every step streams all layers' caches)",
+                   "settle": "2 s idle between building the synthetic caches and the warm-up steps",
                    "replicas": "replicas only" if world > 1 else "single GPU"},
         "phases_us": {"full_verify": statistics.mean(full_ms) * 1e3, "partial_verify": statistics.mean(part_ms) * 1e3,
                       "rest": ms_step * 1e3 - statistics.mean(full_ms) * 1e3 - statistics.mean(part_ms) * 1e3},
