@@ -295,3 +295,37 @@ def run_decode_loop(name, n_steps, period, **over):
             assert int(plens[0]) == o_plen
             pending.extend([0] * len(acc))
     assert o_len > int(c["ctx"][0]) and initialised  # the cache has grown by the accepted tokens
+
+
+@pytest.mark.parametrize("reduce,score_mode", [(0, 0), (1, 0), (2, 0), (0, 1)])
+def test_block_scores_repeat_bit_for_bit_under_back_to_back_launches(reduce, score_mode):
+    """The score kernel's CTAs each walk a share of all tiles with several warps that meet only on shared-memory
+    barriers; a barrier phase that one of them missed shows up as a rare wrong tile, not as a steady error.  Thirty
+    back-to-back launches on the ragged batch-4 shape (shares that cross heads, sequences and layers; 8 layers) must
+    give the same bits every time, and the first of them the scores the oracle computes for sampled heads."""
+    dev = torch.device("cuda")
+    w = wl.make_workload("stress_b4", device=dev, n_layers=8)
+    c = w.cfg
+    L, Hkv, d, bs, M, batch = c["n_layers"], c["Hkv"], c["d"], c["bs"], c["M"], w.batch
+    cfg = util.config_for(w, reduce=reduce, score_mode=score_mode)
+    full = util.full_cache(w)
+    ws = B.new_workspace(cfg, L, batch, full.max_seq_len, M)
+    kmax = torch.zeros((L, batch, Hkv, w.max_blocks, d), dtype=torch.bfloat16, device=dev)
+    kmin = torch.zeros_like(kmax)
+    last_query = torch.tensor([0, 3, M - 1, 7], dtype=torch.int32, device=dev)
+    B.specpv_update_block_summaries(cfg, 0, L, full, None, w.max_blocks, kmax, kmin, ws)
+    runs = [torch.full((L, batch, Hkv, w.max_blocks), 7.0, dtype=torch.float32, device=dev) for _ in range(30)]
+    for s in runs:
+        B.specpv_score_blocks(cfg, 0, L, w.q, None, M, last_query, kmax, kmin, full, s, ws)
+    util.sync_status(ws)
+    for i, s in enumerate(runs[1:], 1):
+        assert torch.equal(s, runs[0]), f"launch {i} differs from launch 0"
+    got = runs[0].cpu().numpy()
+    seq_lens = w.seq_lens.cpu().numpy()
+    qn = wl.to_numpy(w.q)
+    for (l, b) in [(0, 0), (3, 1), (7, 3), (5, 2)]:  # the oracle on whole (layer, sequence) pairs, every KV head
+        nb = (int(seq_lens[b]) + bs - 1) // bs
+        want = oracle.block_scores(qn[l, b], util.widen_t(kmax[l, b])[:, :nb], util.widen_t(kmin[l, b])[:, :nb], Hkv, reduce=reduce,
+                                   last_query=int(last_query[b]), score_mode=score_mode)
+        np.testing.assert_allclose(got[l, b, :, :nb], want, rtol=2e-3, atol=2e-2, err_msg=f"scores l{l} b{b}")
+        assert np.all(got[l, b, :, nb:] == 7.0), "blocks past the context must be left alone"
