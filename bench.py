@@ -295,6 +295,8 @@ def per_layer_graph(st, iters=10):
     res = {}
     for name, cache in (("full_verify_us", st["full"]), ("partial_verify_us", st["partial"])):
         fn = B.specpv_verify_full if name.startswith("full") else B.specpv_verify_partial
+        torch.cuda.synchronize(dev)
+        time.sleep(1.0)  # the partial pass is not measured on a device still warm from the full one
 
         def one_pass():
             for l in range(L):
@@ -455,7 +457,7 @@ def offloaded_refresh(st, layers=4, iters=3):
 def score_variants(st, peaks, iters=10):
     """Block scoring and selection in their variants (Eq. 3's reductions mean / max / last, Eq. 2 as printed and in
     its channel-wise form, selection per head and shared by the heads), each call alone over all layers.  Scoring
-    reads the summaries once: `frac` is against the HBM time of those bytes.  Measured after a one-second pause."""
+    reads the summaries once: `frac` is against the HBM time of those bytes."""
     B, w, L, M, batch = st["B"], st["w"], st["L"], st["M"], st["batch"]
     c = w.cfg
     Hq, Hkv, d, bs = c["Hq"], c["Hkv"], c["d"], c["bs"]
@@ -475,10 +477,6 @@ def score_variants(st, peaks, iters=10):
             b.record()
         torch.cuda.synchronize(dev)
         return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
-    # these are kernel-alone figures (compared with the burst copy rate): let the device settle after the heavy sections
-    # that ran before, which leave it at a power-limited clock for a while
-    torch.cuda.synchronize(dev)
-    time.sleep(1.0)
     scores = torch.zeros_like(st["scores"])
     idx = torch.zeros_like(st["idx"])
     count = torch.zeros_like(st["count"])
@@ -671,6 +669,10 @@ def main():
         if not (enabled and rank == 0 and c["dtype"] == "bf16"):
             return None
         try:
+            # every side measurement starts from a settled device: the section before it leaves the part warm and at a
+            # power-limited clock for a while, which moved these figures by up to a third from run to run
+            torch.cuda.synchronize(dev)
+            time.sleep(1.0)
             return fn(*fn_args)
         except Exception as exc:  # noqa: BLE001
             torch.cuda.synchronize(dev)
@@ -717,7 +719,7 @@ def main():
                    "step": "refresh step (full verify + commit + scores + select + gather) + partial step "
                            "(partial verify + commit)",
                    "l2": "inputs larger than L2 (every step streams all layers' caches)",
-                   "settle": "2 s idle between building the synthetic caches and the warm-up steps",
+                   "settle": "2 s idle between building the synthetic caches and the warm-up steps, 1 s before each side measurement",
                    "replicas": "replicas only" if world > 1 else "single GPU"},
         "phases_us": {"full_verify": statistics.mean(full_ms) * 1e3, "partial_verify": statistics.mean(part_ms) * 1e3,
                       "rest": ms_step * 1e3 - statistics.mean(full_ms) * 1e3 - statistics.mean(part_ms) * 1e3},
