@@ -42,6 +42,9 @@ ACCEPT_LEN = 4  # tokens committed per step: the paper's mean accept length is 3
 NCU_DRAM_BYTES_PER_LAYER = {"llama_128k": (1.075296e9 + 5.433088e6) / 2}
 
 
+NCU_PARTIAL_DRAM_BYTES_PER_LAYER = (35.098e6 + 0.078e6) / 2  # partial verification at a 4096-token budget, same capture
+
+
 def ncu_traffic_bytes(workload: str, n_layers: int):
     per_layer = NCU_DRAM_BYTES_PER_LAYER.get(workload)
     return None if per_layer is None else per_layer * n_layers
@@ -281,7 +284,11 @@ def partial_budget_sweep(st, peaks, budgets=(32, 64, 128), iters=10):
         tokens = int(plens.sum())
         nbytes = L * tokens * Hkv * 2 * d * 2 + L * batch * M * (2 * Hq + 2 * Hkv) * d * 2
         out.append({"budget_tokens": budget * bs, "us": us, "bound_us": nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
-                    "frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6)})
+                    "frac": nbytes / (peaks["hbm_gbs"] * 1e9) / (us * 1e-6), "algorithmic_bytes": nbytes,
+                    # DRAM bytes of the partial launch from the 2-layer ncu capture (profiles/attn_tc_kernel_llama_128k.md),
+                    # scaled by the layers; only the budget that capture ran at has a figure
+                    "traffic": NCU_PARTIAL_DRAM_BYTES_PER_LAYER * L
+                    if budget * bs == 4096 and st["w"].name == "llama_128k" and bs == 64 else None})
         del pk, partial
     return out
 
